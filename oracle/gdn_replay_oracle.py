@@ -38,7 +38,8 @@ The sidecar's write side (anchor_write: destination-table indexed stores, Sectio
 
 Pins (tests/test_oracle_pins.py): exact rational arithmetic on tiny projections, the
 unrolled sum of Eq. 5 by explicit matrix products, closed forms for one-hot and
-orthonormal keys, single-row and overwrite cases, continuation from a cut (of the
+orthonormal keys, single-row and overwrite cases (the single-row closed form and a marker-channel
+test also at H_v != H_k and d_k != d_v, which pin the q | k | v channel split), continuation from a cut (of the
 recurrence, of the convolution with its history, and of a whole layer replayed in two
 pieces against one pass), the contraction bound of the replay error, library convolution /
 activation routines, all 256 e4m3 codes, the state sizes printed in the paper's

@@ -361,6 +361,70 @@ def test_single_row_end_to_end_closed_form():
     assert np.allclose(got_tail[:, 2], z, rtol=2 ** -8)
 
 
+GEOMETRIES_UNEQUAL = [(2, 4, 4, 4), (2, 6, 4, 4), (2, 2, 3, 6), (2, 4, 3, 5)]   # (H_k, H_v, d_k, d_v)
+
+
+@pytest.mark.parametrize("Hk,Hv,dk,dv", GEOMETRIES_UNEQUAL)
+def test_single_row_closed_form_with_unequal_head_counts_and_widths(Hk, Hv, dk, dv):
+    """The one-row closed form with H_v != H_k and d_k != d_v (Appendix A's table: 16/32 and 16/48 heads,
+    widths 96/192): channel offsets are written out here with scalars -- q block H_k d_k wide, k block H_k d_k
+    wide, v block H_v d_v wide, C = 2 H_k d_k + H_v d_v -- and value head h reads key head h // (H_v / H_k)."""
+    r = _rng(150 + Hv * 10 + dv)
+    d = 24
+    C = 2 * Hk * dk + Hv * dv
+    x = torch.from_numpy(r.standard_normal((1, d))).to(torch.bfloat16).double().numpy()
+    W = r.standard_normal((C, d)) / math.sqrt(d)
+    Wab = r.standard_normal((2 * Hv, d)) / math.sqrt(d)
+    cw = r.standard_normal((C, 4))
+    c = r.uniform(0.05, 0.3, Hv); delta = r.uniform(-0.3, 0.3, Hv)
+    S, tail = orc.replay_layer(x, W, Wab, cw, c, delta, n_k_heads=Hk, n_v_heads=Hv, d_k=dk, d_v=dv)
+    assert S.shape == (Hv, dk, dv) and tail.shape == (C, 3)
+    z = [sum(x[0, j] * W[ch, j] for j in range(d)) for ch in range(C)]
+    y = [cw[ch, 3] * z[ch] for ch in range(C)]
+    y = [val / (1 + math.exp(-val)) for val in y]
+    k_block, v_block = Hk * dk, 2 * Hk * dk
+    for h in range(Hv):
+        kh = h // (Hv // Hk)
+        kk = [y[k_block + kh * dk + i] for i in range(dk)]
+        vv = [y[v_block + h * dv + j] for j in range(dv)]
+        nrm = math.sqrt(sum(t * t for t in kk) + 1e-6)
+        b = sum(x[0, j] * Wab[Hv + h, j] for j in range(d))
+        beta = 1 / (1 + math.exp(-b))
+        want = np.array([[beta * (ki / nrm) * vj for vj in vv] for ki in kk])
+        assert np.allclose(S[h], want.astype(np.float32), rtol=2e-7, atol=1e-12), h
+    assert np.allclose(orc.bf16_bits_to_f64(tail)[:, 2], z, rtol=2 ** -8)
+
+
+@pytest.mark.parametrize("Hk,Hv,dk,dv", GEOMETRIES_UNEQUAL)
+def test_marker_channels_land_in_the_right_state_entry(Hk, Hv, dk, dv):
+    """Weights that light up exactly one key channel (key head a, index i) and one value channel (value head h,
+    index j): after one row the only non-zero state entries are S[h'][i][j'] with h' sharing key head a and
+    (h', j') = (h, j).  A key or value offset wrong by one head, or d_v used for d_k, moves or kills the entry."""
+    d = 8
+    C = 2 * Hk * dk + Hv * dv
+    x = np.zeros((1, d)); x[0, 0] = 1.0
+    cw = np.zeros((C, 4)); cw[:, 3] = 1.0
+    Wab = np.zeros((2 * Hv, d))
+    group = Hv // Hk
+    for a in range(Hk):
+        for i in (0, dk - 1):
+            for h in range(Hv):
+                for j in (0, dv - 1):
+                    W = np.zeros((C, d))
+                    W[Hk * dk + a * dk + i, 0] = 2.0              # key channel (a, i)
+                    W[2 * Hk * dk + h * dv + j, 0] = 3.0          # value channel (h, j)
+                    W[a * dk + i, 0] = 5.0                        # the q channel of the same index must not matter
+                    S, tail = orc.replay_layer(x, W, Wab, cw, np.full(Hv, 0.1), np.zeros(Hv), n_k_heads=Hk,
+                                               n_v_heads=Hv, d_k=dk, d_v=dv, activation="identity")
+                    nz = {tuple(idx) for idx in np.argwhere(S != 0)}
+                    want = {(h, i, j)} if h // group == a else set()
+                    assert nz == want, (a, i, h, j, nz)
+                    if want:
+                        assert np.isclose(S[h, i, j], 0.5 * 3.0 * 2.0 / math.sqrt(4.0 + 1e-6), rtol=1e-6)
+                    t = orc.bf16_bits_to_f64(tail)[:, 2]
+                    assert set(np.flatnonzero(t)) == {a * dk + i, Hk * dk + a * dk + i, 2 * Hk * dk + h * dv + j}
+
+
 def test_pipeline_against_library_composition():
     """Whole layer on a small case against torch fp64 library ops (conv1d, silu, normalise)
     feeding a directly written rank-one update loop on torch tensors."""
