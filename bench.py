@@ -8,8 +8,9 @@ conv/SiLU/norm/gates + gated-delta state scan for every rebuilt layer) over one 
 Prints ONE JSON line.  `value` counts layer-tokens (replayed rows x rebuilt layers) per second
 with inputs resident in HBM; `e2e` is the same metric through the host-buffer entry point
 (anchors and tables copied host->device and both states device->host inside the timed region).
-With N > 1 (torchrun) every rank replays its own copy of the batch (requests, layers and heads
-are independent units: no collective on the data path), so the scaling is weak.
+With N > 1 every rank replays its own copy of the batch (requests, layers and heads are independent
+units: no collective on the data path), so the scaling is weak.  Started under torchrun the ranks come
+from the environment; started plainly with --gpus N the script launches its N ranks itself.
 """
 
 import argparse
@@ -27,19 +28,35 @@ METRIC = "replayed tokens/s across linear layers"
 UNIT = "layer-tokens/s"
 DEFAULT_CONFIG = "cfg3"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures whose summaries are committed with the repository (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    # ncu capture of the two-CTA projection on cfg3_slice: 1.780 GB read + 0.635 GB written for 34 880 rows
-    "cfg3_slice": 2.415e9,
-    # the same capture scaled by rows (254 400 / 34 880; 65 536 / 34 880 for cfg2, same widths): upper bounds,
-    # the weight part of the reads does not grow with rows
-    "cfg3": 17.6e9,
-    "cfg2": 4.54e9,
-    # ncu capture of the same kernel on fp16-staged operands, cfg4_slice: 1.505 GB + 0.592 GB for 32 768 rows; cfg4 has 262 144
-    "cfg4_slice": 2.098e9,
-    "cfg4": 16.8e9,
+# Where the DRAM traffic of the dominant kernel comes from: the committed summary of an ncu capture of that
+# kernel on a slice of the workload (same kernel, tile shapes and per-row traffic, small enough to capture).
+# Each summary carries one line `traffic_per_launch: read_bytes=... write_bytes=... rows=...`; the figure
+# reported here is that capture scaled by rows (an upper bound: the weight part of the reads does not grow).
+NCU_TRAFFIC_SUMMARY = {
+    "cfg3": "sr_proj_fused2_kernel_cfg3_slice.md", "cfg3_slice": "sr_proj_fused2_kernel_cfg3_slice.md",
+    "cfg2": "sr_proj_fused2_kernel_cfg3_slice.md",
+    "cfg4": "sr_proj_fused2_kernel_fp8_cfg4_slice.md", "cfg4_slice": "sr_proj_fused2_kernel_fp8_cfg4_slice.md",
 }
+
+
+def ncu_traffic(config, rows):
+    """(bytes per launch, source) from the committed ncu summary for `config`, scaled to `rows`; (None, None) if
+    no capture of that kernel shape exists."""
+    import re
+    name = NCU_TRAFFIC_SUMMARY.get(config)
+    if name is None:
+        return None, None
+    path = os.path.join(ROOT, "profiles", name)
+    try:
+        text = open(path).read()
+    except OSError:
+        return None, None
+    m = re.search(r"traffic_per_launch:\s*read_bytes=([0-9.eE+]+)\s+write_bytes=([0-9.eE+]+)\s+rows=(\d+)", text)
+    if not m:
+        return None, None
+    cap_rows = int(m.group(3))
+    total = float(m.group(1)) + float(m.group(2))
+    return total * rows / cap_rows, f"profiles/{name} ({cap_rows} rows captured, scaled by rows to {rows})"
 
 
 def measured_peaks():
@@ -130,31 +147,23 @@ def oracle_one(wl, req, layer, rows):
     return dt
 
 
-def oracle_sample(wl, limit_s=12.0):
-    """A bounded sample of the workload for the CPU oracle: whole (request, layer) units, longest
-    requests first, until about `limit_s` seconds of CPU work (a short calibration run sizes it).
-    Returns (seconds, layer_tokens, description, threads)."""
+ORACLE_JOB_ROWS = 4096
+
+
+def oracle_job(wl, reps=1):
+    """The fixed job the CPU oracle is timed on, the same for every caller: the first min(R, 4096) rows of the
+    longest request, first rebuilt layer, all heads.  Returns (seconds, layer_tokens, description, threads)."""
     s = wl.spec
     lens = wl.replay_lens.cpu().tolist()
-    order = sorted(range(len(lens)), key=lambda i: -lens[i])
     layer = next(l for l, m in enumerate(wl.layer_mask) if m)
-    if not lens or lens[order[0]] <= 0:
+    if not lens or max(lens) <= 0:
         return 1e-9, 0, f"{s.name}: empty batch", _oracle_threads()
-    cal_rows = min(lens[order[0]], 128)
-    per_row = oracle_one(wl, order[0], layer, cal_rows) / cal_rows
-    total_t, total_rows, units = 0.0, 0, []
-    for req in order:
-        if lens[req] <= 0 or total_t >= limit_s:
-            break
-        rows = int(min(lens[req], max(64, (limit_s - total_t) / per_row)))
-        total_t += oracle_one(wl, req, layer, rows)
-        total_rows += rows
-        units.append(f"req {req}: {rows}/{lens[req]} rows")
-        if len(units) >= 16:
-            break
-    desc = (f"{s.name}: layer {layer}, all {s.n_v_heads} heads, " + "; ".join(units) +
-            f" (of {len(lens) * wl.n_active_layers} request-layers in a step)")
-    return total_t, total_rows, desc, _oracle_threads()
+    req = max(range(len(lens)), key=lambda i: (lens[i], -i))
+    rows = int(min(lens[req], ORACLE_JOB_ROWS))
+    total_t = sum(oracle_one(wl, req, layer, rows) for _ in range(reps))
+    desc = (f"{s.name}: request {req} (the longest, {lens[req]} rows), its first {rows} rows, layer {layer}, all "
+            f"{s.n_v_heads} heads, {reps}x (of {len(lens) * wl.n_active_layers} request-layers in a step)")
+    return total_t, rows * reps, desc, _oracle_threads()
 
 
 def max_over_ranks(value, device):
@@ -177,6 +186,39 @@ def shard_units(units, rank, world):
     return list(units[rank::world])
 
 
+def launch_ranks(n, argv):
+    """Re-runs this script as `n` ranks on this node (one per GPU) under torch.distributed.run; returns its exit code."""
+    import socket
+    import subprocess
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def run_dry(args, rank, world):
+    """The multi-rank plumbing without the kernels: rendezvous, barrier, max over ranks, one line from rank 0."""
+    import torch
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group(args.backend)
+        dist.barrier()
+    dev = torch.device("cpu")
+    total_ms = max_over_ranks(args.steps * (10.0 + rank), dev)          # the slowest rank's clock counts
+    value = aggregate_throughput(1000, args.steps, total_ms, world)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                          "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+                          "scaling": "weak", "dry": True, "data": "none",
+                          "config": {"workload": args.config, "note": "dry run: no kernel was launched"}}), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def run_reference(args, rank):
     """--impl reference: the CPU oracle timed on the host cores, same metric and config."""
     if rank != 0:
@@ -187,12 +229,11 @@ def run_reference(args, rank):
     # of minutes); the oracle then reads the pages it samples back to the host and runs on the host cores
     gen_device = "cuda:0" if torch.cuda.is_available() else "cpu"
     wl = synth.build_workload(args.config, device=gen_device)
-    per_step = max(0.5, min(12.0, 120.0 / max(1, args.steps + args.warmup)))
     for _ in range(args.warmup):
-        oracle_sample(wl, limit_s=min(per_step, 1.0))
+        oracle_job(wl)
     total_t, total_lt, desc, threads = 0.0, 0, "", 1
     for _ in range(args.steps):
-        dt, lt, desc, threads = oracle_sample(wl, limit_s=per_step)
+        dt, lt, desc, threads = oracle_job(wl)
         total_t += dt
         total_lt += lt
     value = total_lt / total_t
@@ -200,7 +241,7 @@ def run_reference(args, rank):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.config, "note": "CPU oracle on a bounded sample per step"},
+        "config": {"workload": args.config, "note": "CPU oracle, one fixed bounded job per step (see cpu_baseline.sample)"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -217,14 +258,25 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"],
+                    help="process-group backend for the timing barrier and the max over ranks")
+    ap.add_argument("--dry", action="store_true",
+                    help="launch and reduce only: every rank reports a made-up step time instead of running the "
+                         "kernels (checks the N-rank plumbing on a box without GPUs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not started by a launcher: start one rank per GPU ourselves and let rank 0 print the line
+        raise SystemExit(launch_ranks(args.gpus, sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.dry:
+        run_dry(args, rank, world)
         return
 
     import torch
@@ -237,7 +289,7 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+        dist.init_process_group(args.backend, device_id=dev if args.backend == "nccl" else None)
     if rank == 0:
         sr_build.build()
     if world > 1:
@@ -402,7 +454,7 @@ def main():
     single_ms = sorted(single)[len(single) // 2]
     single_rows = int(lens_saved[longest].item())
 
-    # short steps only: the same call captured once in a CUDA graph and replayed (Section 5.3: replay graphs)
+    # short steps only: the same call captured once in a CUDA graph and replayed (Section 6, "Replay graphs")
     graph_ms = None
     if ms_per_step < 5.0:
         cap = torch.cuda.Stream(dev)
@@ -426,13 +478,14 @@ def main():
         graph_ms = sorted(gt)[len(gt) // 2]
         del g
 
+    traffic, traffic_source = ncu_traffic(args.config, wl.total_rows)
     roofline = {
         "kernel": "projection (anchor gather + in-projection), per layer launch",
         "bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
         "frac": achieved_tf / peak_tf if achieved_tf else None,
         "peak_source": f"{peaks['source']} bf16 {'sustained' if long_step else 'burst'}",
         "flops_per_launch": proj_flops_per_lt * wl.total_rows,
-        "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.config),
+        "traffic": traffic, "traffic_source": traffic_source,
         "kernel_ms": kernel_ms, "kernel_time_share": kernel_share,
         "scan": {"kernels": "chunk-local + state chain, per layer", "achieved": scan_tf, "unit": "TFLOP/s",
                  "frac": scan_tf / peak_tf if scan_tf else None, "flops_per_layer_token": scan_flops_per_lt,
@@ -478,7 +531,7 @@ def main():
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        dt, lt, desc, threads = oracle_sample(wl, limit_s=12.0)
+        dt, lt, desc, threads = oracle_job(wl, reps=2)
         cpu_baseline = {"value": lt / dt, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
                         "seconds": dt}
 
@@ -487,7 +540,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             # operand type of the tensor-core products: bf16, or fp16 for block-scaled weights (dequantised to fp16)
-            "dtype": "f16" if (spec.weight_format == "e4m3_block128" and os.environ.get("SR_FP8_EXACT") != "1") else "bf16",
+            "dtype": "f16" if spec.weight_format == "e4m3_block128" else "bf16",
             "data": "synthetic",
             "config": {"workload": spec.name, "n_layers_rebuilt": wl.n_active_layers, "d_model": spec.d_model,
                        "heads": spec.n_v_heads, "d_head": spec.d_k, "requests": spec.n_requests,

@@ -4,7 +4,7 @@
  * The library rebuilds the recurrent state of gated-delta-rule linear-attention layers
  * at a matched prefix-cache page boundary by replaying only the retained anchor hidden
  * states of a recent suffix, from a zero state (paper Eq. 2, "S'_j = f(h_{j-k+1..j})"),
- * for a packed batch of cache hits with different replay lengths (Section 5.3,
+ * for a packed batch of cache hits with different replay lengths (Section 5.2,
  * "Batched replay").  It writes, per (request, rebuilt layer), the two pieces of state a
  * linear-attention layer carries across tokens (Appendix A, "Native cache"):
  *
@@ -36,7 +36,7 @@
  *   - every call returns an sr_status; problems detectable on the host are reported
  *     before anything is launched.  Problems only visible on the device (a page id outside
  *     the pool, a replay length outside [0, max_replay_len]) follow the paper's fail-closed
- *     rule (Section 5.3: a hit that cannot be served is treated as a miss): that request is
+ *     rule (Section 5.2: a hit that cannot be served is treated as a miss): that request is
  *     skipped, its outputs are left untouched, and a bit is set in a device status word
  *     readable with sr_device_status.  No kernel traps or spins without bound.
  */
@@ -63,9 +63,10 @@ typedef enum sr_status {
 /* bits of the device status word (sr_device_status) */
 #define SR_DEV_BAD_REPLAY_LEN 0x1u /* some replay_lens[i] < 0 or > max_replay_len      */
 #define SR_DEV_BAD_PAGE_ID 0x2u    /* some used page-table entry outside [0, n_phys)   */
-#define SR_DEV_BAD_SLOT 0x4u       /* some state_slots[i] < -1                          */
+#define SR_DEV_BAD_SLOT 0x4u       /* some state_slots[i] < -1, or >= n_state_slots      */
 #define SR_DEV_ROWS_OVERFLOW 0x8u  /* sum of replay lengths above max_total_rows        */
 #define SR_DEV_WAIT_EXPIRED 0x10u  /* a bounded in-kernel wait gave up (internal fault) */
+#define SR_DEV_BOUNDS_CHECK 0x20u  /* SR_DEBUG_CHECK_BOUNDS only: an index left its array  */
 
 enum { SR_W_BF16 = 0, SR_W_E4M3_BLOCK128 = 1 };   /* sr_model_desc.weight_format   */
 enum { SR_CONV_SILU = 0, SR_CONV_IDENTITY = 1 };  /* sr_model_desc.conv_activation */
@@ -73,6 +74,18 @@ enum { SR_CONV_SILU = 0, SR_CONV_IDENTITY = 1 };  /* sr_model_desc.conv_activati
  * GATED_DELTA: A_t(S) = alpha_t (I - beta_t k_t k_t^T) S.  DECAY_ONLY: A_t(S) = alpha_t S (per-head decay, no
  * erase).  The write B_t = beta_t k_t v_t^T and everything before the recurrence are the same. */
 enum { SR_REC_GATED_DELTA = 0, SR_REC_DECAY_ONLY = 1 };
+
+/* sr_model_desc.debug_flags: switches for tests and diagnostics.  They select a second form of one step (to
+ * test it against the same oracle) or add checks; results stay within the documented tolerances. */
+#define SR_DEBUG_DOT_CONV_STATE 0x1u /* conv state by per-channel dot products instead of the batched GEMM       */
+#define SR_DEBUG_SINGLE_CTA_MMA 0x2u /* projection on one-CTA MMA tiles where CTA pairs would be used             */
+#define SR_DEBUG_FP8_EXACT 0x4u      /* e4m3 weights: fp32 promotion of bare-code partial sums, no 16-bit staging */
+#define SR_DEBUG_CHECK_BOUNDS 0x8u   /* kernels range-check every table-driven index before the access, skip the
+                                        access and record SR_DEV_BOUNDS_CHECK instead of reading or writing       */
+#define SR_DEBUG_EXPIRE_WAIT 0x10u   /* fault-injection for the bounded waits: the state chain's first in-kernel
+                                        wait is given a limit of about a millisecond and the arrival it waits for
+                                        is withheld, so the wait gives up, SR_DEV_WAIT_EXPIRED is raised, the
+                                        affected outputs stay untouched and the kernel returns normally          */
 
 /* Model geometry, HOST struct, fixed at sr_create.  Sizes follow Appendix A's notation. */
 typedef struct sr_model_desc {
@@ -88,6 +101,7 @@ typedef struct sr_model_desc {
   int32_t conv_activation; /* SR_CONV_*                                                 */
   float l2_eps;            /* epsilon inside the key normalisation (1e-6)               */
   int32_t recurrence;      /* SR_REC_* (0 = gated delta rule)                           */
+  uint32_t debug_flags;    /* SR_DEBUG_* test and diagnostic switches; 0 in production  */
 } sr_model_desc;
 
 /* One layer's parameters: HOST struct holding DEVICE pointers.  The array handed to
@@ -116,7 +130,7 @@ typedef struct sr_anchor_pool {
   const int32_t* layer_to_pool;  /* HOST [n_layers]: pool layer of each model layer, -1 = none */
 } sr_anchor_pool;
 
-/* The batch of cache hits (Section 5.3: packed variable-length execution with
+/* The batch of cache hits (Section 5.2: packed variable-length execution with
  * device-side boundaries and destination slots): HOST struct. */
 typedef struct sr_page_table {
   const int32_t* pages;        /* DEVICE [n_requests][max_pages]: physical pages of each request's
@@ -125,13 +139,16 @@ typedef struct sr_page_table {
   const int32_t* state_slots;  /* DEVICE [n_requests] or NULL (= request index).  Destination slot
                                   in the outputs; -1 is the sentinel of a padding segment: nothing is
                                   read or written for it and no status bit is set */
-  int32_t n_requests;
+  int32_t n_requests;          /* at most 65535 (one grid row per request), else SR_ERR_UNSUPPORTED_SHAPE */
   int32_t max_pages;           /* second extent of `pages` */
   int32_t max_replay_len;      /* upper bound on every replay_lens[i] (<= max_pages*page_rows) */
   int64_t max_total_rows;      /* upper bound on the sum of replay_lens (sizes grid and workspace); with
                                   d_k = d_v = 128 at most 65535 page slots per call, i.e.
                                   max_total_rows / 64 + n_requests <= 65535 (about 4.19 M rows), else
                                   SR_ERR_UNSUPPORTED_SHAPE */
+  int32_t n_state_slots;       /* slots the output arrays hold, or 0 = not stated.  When stated, a destination
+                                  slot >= n_state_slots is treated like any other invalid request (skipped,
+                                  SR_DEV_BAD_SLOT) instead of being written through */
 } sr_page_table;
 
 /* An output array: slot s, layer l starts at base + s*slot_stride + l*layer_stride. */
@@ -171,7 +188,7 @@ int sr_workspace_bytes(const sr_ctx* ctx, const sr_page_table* table, size_t* ou
 
 /*
  * Rebuilds the recurrent and conv state of every layer l with layer_mask[l] != 0 for every
- * request of the batch (Eq. 2 and Eq. 4; Section 5.3 for the batch form).
+ * request of the batch (Eq. 2 and Eq. 4; Section 5.2 for the batch form).
  *
  *   replay_lens  DEVICE [n_requests] int32: rows to replay per request (any value >= 0;
  *                0 gives a zero state and a zero conv state)
@@ -208,7 +225,9 @@ int sr_replay_states(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_tabl
  *     sr_workspace_bytes) the call returns SR_ERR_WORKSPACE and launches nothing.  128 MiB covers,
  *     for example, 4096 packed rows in 8 requests at d_k = d_v = 128 with 16 key / 32 value heads;
  *   - the first call on each device looks up the array's device address (with that device
- *     current); make that first call outside any stream capture;
+ *     current).  With CUDA's lazy module loading that look-up is also the moment the array is
+ *     materialised on the device: make one call at start-up, outside any stream capture and before the
+ *     process freezes or fills its device memory; later calls leave the device's free memory unchanged;
  *   - the call allocates nothing: no cudaMalloc, no cudaFree, no allocating library routine;
  *   - all calls on a device share the one array, and it keeps whatever the previous call left.
  *     Nothing in it needs to start at zero (each call rewrites what it reads), but two calls whose
@@ -246,7 +265,7 @@ int sr_replay_states_from(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page
                           size_t workspace_bytes, void* stream);
 
 /*
- * The same call for a caller whose anchors live in a host pool (Section 5.3: anchors are
+ * The same call for a caller whose anchors live in a host pool (Section 5.2: anchors are
  * fetched with asynchronous host-to-device copies before replay): copies the HOST
  * anchor pool, page table, slots and replay lengths into the caller's DEVICE staging
  * buffers, runs sr_replay_states on them, and copies both outputs back to HOST memory;
@@ -272,7 +291,7 @@ int sr_replay_states_host(sr_ctx* ctx, const void* host_pool, size_t pool_bytes,
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * The write side of the sidecar (Section 5.2, "Writing anchors": the host precomputes a
+ * The write side of the sidecar (Section 5.1, "Writing anchors": the host precomputes a
  * destination table for the step; indexed copies inside the step's graph write the selected
  * hidden states directly to their sidecar locations; unsampled positions receive a scratch
  * address and are ignored).  For every token t with dest_page[t] >= 0 and every i < n_layers:
@@ -312,7 +331,7 @@ int sr_device_status(sr_ctx* ctx, const void* workspace, void* stream, uint32_t*
 /* Number of kernels the last sr_replay_states / sr_debug_gather call on `ctx` launched. */
 int sr_last_launch_count(const sr_ctx* ctx, int64_t* out_launches);
 
-/* Kernel kinds of the replay path, in launch order per layer (Section 5.3's replay executes
+/* Kernel kinds of the replay path, in launch order per layer (Section 5.2's replay executes
  * "the computation needed to reconstruct each group"; these are its parts). */
 enum {
   SR_KERNEL_SCHEDULE = 0,   /* batch packing, once per call                          */

@@ -34,7 +34,7 @@ the functions below are pinned by tests, the *choices* are "parity unpinned"):
     projections; value head h uses key head h // (H_v / H_k);
   * the conv state lists, per channel, the last w-1 projection rows oldest first.
 
-The sidecar's write side (anchor_write: destination-table indexed stores, Section 5.2) is restated too.
+The sidecar's write side (anchor_write: destination-table indexed stores, Section 5.1) is restated too.
 
 Pins (tests/test_oracle_pins.py): exact rational arithmetic on tiny projections, the
 unrolled sum of Eq. 5 by explicit matrix products, closed forms for one-hot and
@@ -114,7 +114,7 @@ def gather_anchor_rows(pool, pages, n_rows: int, pool_layer: int, page_rows: int
 
 
 def anchor_write(pool, hidden_bits, dest_page, dest_row, pool_layer: int) -> None:
-    """The write side of the sidecar (Section 5.2, "Writing anchors"): token t of a step stores its hidden state
+    """The write side of the sidecar (Section 5.1, "Writing anchors"): token t of a step stores its hidden state
     at row dest_row[t] of page dest_page[t]; a negative page is the scratch address -- the token is not sampled
     and nothing is stored.  `pool` is a uint16 array [n_phys, L_pool, page_rows, d], updated in place;
     `hidden_bits` uint16 [n_tokens, d]."""

@@ -23,6 +23,8 @@ SR_DEV_BAD_REPLAY_LEN, SR_DEV_BAD_PAGE_ID, SR_DEV_BAD_SLOT, SR_DEV_ROWS_OVERFLOW
 SR_W_BF16, SR_W_E4M3_BLOCK128 = 0, 1
 SR_CONV_SILU, SR_CONV_IDENTITY = 0, 1
 SR_REC_GATED_DELTA, SR_REC_DECAY_ONLY = 0, 1
+SR_DEV_BOUNDS_CHECK = 32
+SR_DEBUG_DOT_CONV_STATE, SR_DEBUG_SINGLE_CTA_MMA, SR_DEBUG_FP8_EXACT, SR_DEBUG_CHECK_BOUNDS, SR_DEBUG_EXPIRE_WAIT = 1, 2, 4, 8, 16
 
 EXPORTS = (
     "sr_version", "sr_status_string", "sr_create", "sr_destroy", "sr_ssm_bytes_per_layer",
@@ -39,7 +41,8 @@ class sr_model_desc(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_k_heads", C.c_int32),
                 ("n_v_heads", C.c_int32), ("d_k", C.c_int32), ("d_v", C.c_int32),
                 ("conv_width", C.c_int32), ("page_rows", C.c_int32), ("weight_format", C.c_int32),
-                ("conv_activation", C.c_int32), ("l2_eps", C.c_float), ("recurrence", C.c_int32)]
+                ("conv_activation", C.c_int32), ("l2_eps", C.c_float), ("recurrence", C.c_int32),
+                ("debug_flags", C.c_uint32)]
 
 
 class sr_layer_weights(C.Structure):
@@ -55,7 +58,8 @@ class sr_anchor_pool(C.Structure):
 
 class sr_page_table(C.Structure):
     _fields_ = [("pages", C.c_void_p), ("state_slots", C.c_void_p), ("n_requests", C.c_int32),
-                ("max_pages", C.c_int32), ("max_replay_len", C.c_int32), ("max_total_rows", C.c_int64)]
+                ("max_pages", C.c_int32), ("max_replay_len", C.c_int32), ("max_total_rows", C.c_int64),
+                ("n_state_slots", C.c_int32)]
 
 
 class sr_out(C.Structure):
@@ -223,11 +227,12 @@ def sr_profile_read(ctx, kind: int):
 
 # ---- marshalling of torch tensors ---------------------------------------------------
 
-def model_desc(spec, conv_activation: int = SR_CONV_SILU, l2_eps: float = 1e-6) -> sr_model_desc:
+def model_desc(spec, conv_activation: int = SR_CONV_SILU, l2_eps: float = 1e-6, debug_flags: int = 0) -> sr_model_desc:
     fmt = SR_W_E4M3_BLOCK128 if spec.weight_format == "e4m3_block128" else SR_W_BF16
     return sr_model_desc(spec.n_layers, spec.d_model, spec.n_k_heads, spec.n_v_heads, spec.d_k, spec.d_v,
                          spec.conv_width, 64, fmt, conv_activation, l2_eps,
-                         SR_REC_DECAY_ONLY if getattr(spec, "recurrence", "gated_delta") == "decay_only" else SR_REC_GATED_DELTA)
+                         SR_REC_DECAY_ONLY if getattr(spec, "recurrence", "gated_delta") == "decay_only" else SR_REC_GATED_DELTA,
+                         debug_flags)
 
 
 class Replayer:
@@ -241,11 +246,12 @@ class Replayer:
     def __init__(self, workload, conv_activation: int = SR_CONV_SILU, l2_eps: float = 1e-6,
                  state_slots: Optional[torch.Tensor] = None, n_slots: Optional[int] = None,
                  max_total_rows: Optional[int] = None, max_replay_len: Optional[int] = None,
-                 out_ssm: Optional[torch.Tensor] = None, out_conv: Optional[torch.Tensor] = None):
+                 out_ssm: Optional[torch.Tensor] = None, out_conv: Optional[torch.Tensor] = None,
+                 debug_flags: int = 0):
         self.wl = workload
         spec = workload.spec
         self.spec = spec
-        self.desc = model_desc(spec, conv_activation, l2_eps)
+        self.desc = model_desc(spec, conv_activation, l2_eps, debug_flags)
         self.ctx = sr_create(self.desc)
         dev = workload.page_table.device
         if dev.type != "cuda":
@@ -271,7 +277,7 @@ class Replayer:
             max_replay_len = min(int(max_pages) * 64, max(0, int(lens_host.max().item()) if B else 0))
         self.table = sr_page_table(
             workload.page_table.data_ptr(), state_slots.data_ptr() if state_slots is not None else None,
-            B, max_pages, max_replay_len, max_total_rows)
+            B, max_pages, max_replay_len, max_total_rows, int(n_slots) if n_slots is not None else B)
         self.n_slots = int(n_slots) if n_slots is not None else B
         self.ssm_layer_bytes = sr_ssm_bytes_per_layer(self.ctx)
         self.conv_layer_bytes = sr_conv_bytes_per_layer(self.ctx)

@@ -1,4 +1,4 @@
-// Anchor write path (Section 5.2, "Writing anchors"): the host builds a destination table for the step, and
+// Anchor write path (Section 5.1, "Writing anchors"): the host builds a destination table for the step, and
 // indexed copies inside the step's graph write the selected hidden states straight to their sidecar rows;
 // positions that are not sampled carry a scratch address and are ignored.
 //

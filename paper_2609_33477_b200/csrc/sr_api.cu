@@ -1,10 +1,47 @@
 // The C boundary: argument checking and the per-layer launch sequence.  No arithmetic of the
 // method lives here; every step runs in the kernels the launch functions enqueue.
+#include <mutex>
 #include <new>
 #include <stdlib.h>
 #include <string.h>
 
 #include "sr_common.cuh"
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_device_mutex;
+bool g_once_done[kMaxDevices][SR_ONCE_KEYS];
+int g_sm_count[kMaxDevices];
+}  // namespace
+
+cudaError_t sr_once_per_device(int key, cudaError_t (*setup)()) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices || key < 0 || key >= SR_ONCE_KEYS) return cudaErrorInvalidValue;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  if (g_once_done[dev][key]) return cudaSuccess;
+  e = setup();
+  if (e == cudaSuccess) g_once_done[dev][key] = true;
+  return e;
+}
+
+cudaError_t sr_current_device_sms(int* sms) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidValue;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  if (g_sm_count[dev] <= 0) {
+    int n = 0;
+    e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    if (n <= 0) return cudaErrorInvalidValue;
+    g_sm_count[dev] = n;
+  }
+  *sms = g_sm_count[dev];
+  return cudaSuccess;
+}
 
 namespace {
 
@@ -13,12 +50,13 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 int check_batch(const sr_ctx* ctx, const sr_page_table* t) {
   if (!ctx || !t) return SR_ERR_INVALID_ARG;
   if (!ctx->kernels_cover) return SR_ERR_UNSUPPORTED_SHAPE;
-  if (t->n_requests < 0 || t->max_pages < 0 || t->max_replay_len < 0 || t->max_total_rows < 0) return SR_ERR_INVALID_ARG;
+  if (t->n_requests < 0 || t->max_pages < 0 || t->max_replay_len < 0 || t->max_total_rows < 0 || t->n_state_slots < 0)
+    return SR_ERR_INVALID_ARG;
   if (t->n_requests > 65535) return SR_ERR_UNSUPPORTED_SHAPE;   // one grid row per request
   if ((int64_t)t->max_replay_len > (int64_t)t->max_pages * ctx->desc.page_rows) return SR_ERR_INVALID_ARG;
   if (t->max_total_rows > (int64_t)1 << 30) return SR_ERR_UNSUPPORTED_SHAPE;
   // the tensor-core kernels index page slots with one grid row (and one 32-bit tile coordinate) per slot
-  if (ctx->fused && sr_workspace_layout(ctx, t->n_requests, t->max_pages, t->max_total_rows).max_slots > 65535)
+  if (sr_workspace_layout(ctx, t->n_requests, t->max_pages, t->max_total_rows).max_slots > 65535)
     return SR_ERR_UNSUPPORTED_SHAPE;
   return SR_OK;
 }
@@ -103,32 +141,22 @@ int sr_create(const sr_model_desc* d, sr_ctx** out_ctx) {
   c->n_k = d->n_k_heads * d->d_k;
   c->n_v = d->n_v_heads * d->d_v;
   c->n_gate = 2 * d->n_v_heads;
-  c->n_z = c->n_k + c->n_v + c->n_gate;
-  c->ldz = (c->n_z + 63) / 64 * 64;
   c->conv_ch = 2 * c->n_k + c->n_v;
   c->last_launches = 0;
   c->profiling = false;
   c->ev_used = 0;
-  c->sm_count = 0;
   c->copy_in = nullptr;
   c->copy_out = nullptr;
-  const char* simt = getenv("SR_SIMT_PROJECTION");
-  c->simt_projection = simt && simt[0] == '1';
-  const char* msc = getenv("SR_MMA_SYNC_CHAIN");
-  c->mma_sync_chain = msc && msc[0] == '1';
-  const char* tok = getenv("SR_TOKEN_SCAN");
-  c->token_scan = tok && tok[0] == '1';
+  c->debug_flags = d->debug_flags;
   c->wdec_bytes = 0;
-  c->kernels_cover = sr_scan_token_supported(d->d_k, d->d_v) && d->d_model % 128 == 0 &&
-                     d->conv_width == SR_CONV_W && d->page_rows == SR_PAGE_ROWS;
-  if (c->kernels_cover && !c->simt_projection) c->wdec_bytes = sr_proj_umma_decoded_bytes(c);
-  // the fused format needs the tensor-core projection and the chunk scan; SR_UNFUSED=1 keeps the fp32 scratch path
-  const char* unf = getenv("SR_UNFUSED");
-  c->fused = c->kernels_cover && !c->simt_projection && !c->token_scan && !(unf && unf[0] == '1') &&
-             sr_proj_fused_supported(c) && sr_scan_chunk_supported(c);
-  const char* fpe = getenv("SR_FP8_EXACT");
-  c->fp16_stage = c->fused && d->weight_format == SR_W_E4M3_BLOCK128 && !(fpe && fpe[0] == '1');
-  if (c->fused && d->weight_format == SR_W_E4M3_BLOCK128)
+  c->kernels_cover = d->conv_width == SR_CONV_W && d->page_rows == SR_PAGE_ROWS && sr_proj_fused_supported(c) &&
+                     sr_chunk_local_supported(d->d_k, d->d_v) && sr_scan_chain_supported(d->d_k, d->d_v);
+  const bool e4m3 = d->weight_format == SR_W_E4M3_BLOCK128;
+  // block-scaled weights: fp16 staging by default; fp32 promotion of bare-code partial sums on request, where the
+  // channel tiles line up with the scale blocks
+  c->fp16_stage = c->kernels_cover && e4m3 &&
+                  !((d->debug_flags & SR_DEBUG_FP8_EXACT) && sr_proj_fused_exact_fp8_supported(c));
+  if (c->kernels_cover && e4m3)
     c->wdec_bytes = (size_t)(c->n_k + c->n_v + (c->fp16_stage ? c->n_gate : 0)) * d->d_model * 2;
   *out_ctx = c;
   return SR_OK;
@@ -179,9 +207,8 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
                 const sr_out* out_conv, void* workspace, size_t workspace_bytes, void* stream_,
                 const LayerHooks* hooks, const sr_out* in_ssm = nullptr, const sr_out* in_conv = nullptr) {
   int st = check_batch(ctx, table);
+  if (st != SR_OK) return st;
   if (in_ssm || in_conv) {
-    // continuation is served by the default kernels only
-    if (!ctx->fused || ctx->mma_sync_chain) return SR_ERR_UNSUPPORTED_SHAPE;
     if (in_ssm && (!in_ssm->base || !aligned(in_ssm->base, 16) || in_ssm->slot_stride_bytes % 16 ||
                    in_ssm->layer_stride_bytes % 16))
       return SR_ERR_INVALID_ARG;
@@ -189,7 +216,6 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
                     in_conv->layer_stride_bytes % 2))
       return SR_ERR_INVALID_ARG;
   }
-  if (st != SR_OK) return st;
   if (!replay_lens || !layer_mask || !weights || !out_ssm || !out_conv || !table->pages) return SR_ERR_INVALID_ARG;
   if (!out_ssm->base || !out_conv->base) return SR_ERR_INVALID_ARG;
   if (!aligned(out_ssm->base, 16) || out_ssm->slot_stride_bytes % 16 || out_ssm->layer_stride_bytes % 16)
@@ -218,22 +244,13 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
   const SrSched sched = sr_sched_view(workspace, lay, table->n_requests);
   const SrPoolView pv = pool_view(pool);
   float* z = (float*)((char*)workspace + lay.off_z);
-  if (ctx->sm_count == 0) {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-      return SR_ERR_CUDA;
-    ctx->sm_count = sms;
-  }
-  const bool use_umma = !ctx->simt_projection && sr_proj_umma_supported(ctx);
-  // the decay-only family is served by the default kernels and by the token scan
-  const bool use_chunk_scan = !ctx->token_scan && sr_scan_chunk_supported(ctx) && d.recurrence == SR_REC_GATED_DELTA;
-  if (d.recurrence != SR_REC_GATED_DELTA && ctx->fused && ctx->mma_sync_chain) return SR_ERR_UNSUPPORTED_SHAPE;
+  int sm_count = 0;
+  if (sr_current_device_sms(&sm_count) != cudaSuccess) return SR_ERR_CUDA;
   SrFused fused_buf;
   fused_buf.kv16 = (__half*)((char*)workspace + lay.off_kv16);
   fused_buf.zraw = (float*)((char*)workspace + lay.off_zraw);
   fused_buf.gates = z;
-  fused_buf.ncb = (ctx->n_k + ctx->n_v) / 128;
+  fused_buf.ncb = (ctx->n_k + ctx->n_v + 127) / 128;
   fused_buf.n_kv = ctx->n_k + ctx->n_v;
   fused_buf.n_gate = ctx->n_gate;
   fused_buf.fix_mod = (d.weight_format == SR_W_E4M3_BLOCK128 && !ctx->fp16_stage) ? 2 : 4;
@@ -242,12 +259,13 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
   fused_buf.in_ssm_slot_stride = 0;
   fused_buf.x16 = ctx->fp16_stage ? (const __half*)((char*)workspace + lay.off_x16) : nullptr;
   fused_buf.w16 = ctx->fp16_stage ? (const __half*)((char*)workspace + lay.off_wdec) : nullptr;
-  const SrFused* fused = ctx->fused ? &fused_buf : nullptr;
+  const SrFused& fused = fused_buf;
 
   {
     LaunchScope scope(ctx, stream, SR_KERNEL_SCHEDULE);
     if (sr_launch_schedule(sched, table->pages, table->state_slots, replay_lens, table->max_pages,
-                           table->max_replay_len, table->max_total_rows, pool->n_phys_pages, stream) != cudaSuccess)
+                           table->max_replay_len, table->max_total_rows, pool->n_phys_pages, table->n_state_slots,
+                           stream) != cudaSuccess)
       return SR_ERR_CUDA;
   }
   for (int l = 0; l < d.n_layers; ++l) {
@@ -277,46 +295,31 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
       LaunchScope scope(ctx, stream, SR_KERNEL_ANCHOR_STAGE);
       if (sr_launch_stage_anchors_fp16(ctx, sched, pv, pl, (__half*)((char*)workspace + lay.off_x16), stream) != cudaSuccess)
         return SR_ERR_CUDA;
-    } else if ((use_umma || fused) && ctx->wdec_bytes) {
+    } else if (ctx->wdec_bytes) {
       LaunchScope scope(ctx, stream, SR_KERNEL_WEIGHT_DECODE);
       if (sr_launch_weight_decode(ctx, weights[l], wdec, stream) != cudaSuccess) return SR_ERR_CUDA;
     }
     {
       LaunchScope scope(ctx, stream, SR_KERNEL_PROJECTION);
-      cudaError_t e;
-      if (fused)
-        e = sr_launch_proj_fused(ctx, sched, *pool, pl, weights[l], ctx->wdec_bytes ? wdec : nullptr, *fused,
-                                 ctx->sm_count, stream);
-      else if (use_umma)
-        e = sr_launch_proj_umma(ctx, sched, *pool, pl, weights[l], ctx->wdec_bytes ? wdec : nullptr, z, ctx->sm_count,
-                                stream);
-      else
-        e = sr_launch_proj_simt(ctx, sched, pv, pl, weights[l], z, stream);
-      if (e != cudaSuccess) return SR_ERR_CUDA;
+      if (sr_launch_proj_fused(ctx, sched, *pool, pl, weights[l], ctx->wdec_bytes ? wdec : nullptr, fused, sm_count,
+                               stream) != cudaSuccess)
+        return SR_ERR_CUDA;
     }
     {
       LaunchScope scope(ctx, stream, SR_KERNEL_CONV_TAIL, sr_conv_tail_launches(ctx));
-      if (sr_launch_conv_tail(ctx, sched, pv, pl, weights[l], z, fused, conv_l, out_conv->slot_stride_bytes, stream) !=
+      if (sr_launch_conv_tail(ctx, sched, pv, pl, weights[l], fused, conv_l, out_conv->slot_stride_bytes, stream) !=
           cudaSuccess)
         return SR_ERR_CUDA;
     }
-    if (fused) {
+    {
       void* split = (char*)workspace + lay.off_split;
       {
         LaunchScope scope(ctx, stream, SR_KERNEL_CHUNK_LOCAL);
-        if (sr_launch_chunk_local(ctx, sched, weights[l], *fused, split, stream) != cudaSuccess) return SR_ERR_CUDA;
+        if (sr_launch_chunk_local(ctx, sched, weights[l], fused, split, stream) != cudaSuccess) return SR_ERR_CUDA;
       }
       LaunchScope scope(ctx, stream, SR_KERNEL_SCAN);
-      const cudaError_t e =
-          ctx->mma_sync_chain ? sr_launch_scan_chain(ctx, sched, *fused, split, ssm_l, out_ssm->slot_stride_bytes, stream)
-                              : sr_launch_scan_chain_umma(ctx, sched, *fused, split, ssm_l, out_ssm->slot_stride_bytes, stream);
-      if (e != cudaSuccess) return SR_ERR_CUDA;
-    } else {
-      LaunchScope scope(ctx, stream, SR_KERNEL_SCAN);
-      const cudaError_t e = use_chunk_scan
-                                ? sr_launch_scan_chunk(ctx, sched, weights[l], z, ssm_l, out_ssm->slot_stride_bytes, stream)
-                                : sr_launch_scan_token(ctx, sched, weights[l], z, ssm_l, out_ssm->slot_stride_bytes, stream);
-      if (e != cudaSuccess) return SR_ERR_CUDA;
+      if (sr_launch_scan_chain_umma(ctx, sched, fused, split, ssm_l, out_ssm->slot_stride_bytes, sm_count, stream) != cudaSuccess)
+        return SR_ERR_CUDA;
     }
     if (hooks && !hooks->after(hooks->user, l, stream)) return SR_ERR_CUDA;
   }
@@ -552,7 +555,8 @@ int sr_debug_gather(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table
   ctx->ev_used = 0;
   ctx->ev_kind.clear();
   if (sr_launch_schedule(sched, table->pages, table->state_slots, replay_lens, table->max_pages,
-                         table->max_replay_len, table->max_total_rows, pool->n_phys_pages, stream) != cudaSuccess)
+                         table->max_replay_len, table->max_total_rows, pool->n_phys_pages, table->n_state_slots,
+                           stream) != cudaSuccess)
     return SR_ERR_CUDA;
   if (sr_launch_debug_gather(sched, pool_view(pool), pool->layer_to_pool[layer], ctx->desc.d_model, table->max_pages,
                              out_rows, out_capacity_rows, stream) != cudaSuccess)

@@ -21,20 +21,14 @@ struct sr_ctx {
   int n_k;        // H_k * d_k   (key columns of the projection)
   int n_v;        // H_v * d_v   (value columns)
   int n_gate;     // 2 * H_v     (decay and write-strength columns)
-  int n_z;        // n_k + n_v + n_gate: columns the scan needs from the projection
-  int ldz;        // row pitch of the projection scratch in floats
   int conv_ch;    // C = 2 H_k d_k + H_v d_v
   int64_t last_launches;
   bool kernels_cover;  // false: sizes can be queried but no kernel serves this geometry
   size_t wdec_bytes;   // workspace bytes for decoded e4m3 codes (0 for bf16 weights)
-  bool fused;          // projection epilogue applies conv + SiLU and hands fp16 k, v tiles to the chunk scan
   bool fp16_stage;     // block-scaled weights on the fused path: weights dequantised and anchors converted to fp16
-                       // once per layer, then the same tensor-core kernel as for bf16 weights (environment
-                       // SR_FP8_EXACT=1 selects fp32 promotion of bare-code partial sums instead)
-  int sm_count;        // SMs of the device the first launching call ran on (0 = not asked yet)
-  bool mma_sync_chain;   // debugging aid (environment SR_MMA_SYNC_CHAIN=1): state chain on mma.sync instead of tcgen05
-  bool token_scan;       // debugging aid (environment SR_TOKEN_SCAN=1): token-by-token scan instead of the chunked one
-  bool simt_projection;  // debugging aid (environment SR_SIMT_PROJECTION=1): keep the projection off the tensor cores
+                       // once per layer, then the same tensor-core kernel as for bf16 weights (SR_DEBUG_FP8_EXACT
+                       // selects fp32 promotion of bare-code partial sums instead)
+  uint32_t debug_flags;  // desc.debug_flags (SR_DEBUG_*)
   // optional per-kernel timing (sr_profile_*): events bracketing every launch of the last call
   bool profiling;
   std::vector<cudaEvent_t> ev_pool;   // created on demand, reused, destroyed with the context
@@ -44,6 +38,17 @@ struct sr_ctx {
   std::vector<int> ev_kind;           // kernel kind of bracket i (events 2i, 2i+1)
   size_t ev_used;
 };
+
+// Per-device one-time set-up (kernel attributes are per device, and several host threads may make their first
+// call at once): runs `setup` with the current device the first time `key` is seen on it, under a lock; later
+// calls return cudaSuccess at once.  A failed set-up is retried by the next call.
+enum SrOnceKey {
+  SR_ONCE_PROJ_FUSED = 0, SR_ONCE_PROJ_FUSED2, SR_ONCE_CHUNK_LOCAL_64, SR_ONCE_CHUNK_LOCAL_96,
+  SR_ONCE_CHUNK_LOCAL_128, SR_ONCE_CHAIN_UMMA, SR_ONCE_KEYS
+};
+cudaError_t sr_once_per_device(int key, cudaError_t (*setup)());
+// SM count of the current device (looked up once per device)
+cudaError_t sr_current_device_sms(int* sms);
 
 // Scratch layout inside the caller's workspace (all offsets in bytes, 256-aligned).
 struct sr_ctx;
@@ -59,13 +64,13 @@ struct SrWorkspace {
   size_t off_slot_page;  // int32 [max_slots] physical page of each page slot
   size_t off_slot_rows;  // int32 [max_slots] valid rows in the slot (1..64)
   size_t off_slot_first; // int32 [max_slots] request index + 1 where the slot opens its request, else 0
-  size_t off_kv16;       // fused: half [max_slots][(n_k+n_v)/128][64][128] conv + SiLU outputs, one layer at a time
-  size_t off_zraw;       // fused: float [max_slots][6][n_k+n_v] raw projection rows 0,1,2 | last 3 valid
-  size_t off_z;          // float [max_slots*64][ldz] projection scratch, one layer at a time
-  size_t off_split;      // fused: per (slot, head) T matrices (fp16) and row factors handed from the chunk-local
+  size_t off_kv16;       // half [max_slots][ncb * 128][64] conv + SiLU outputs, one layer at a time
+  size_t off_zraw;       // float [max_slots][6][n_k+n_v] raw projection rows 0,1,2 | last 3 valid
+  size_t off_z;          // float [max_slots][2 H_v][64] raw gate pre-activations, one layer at a time
+  size_t off_split;      // per (slot, head) T matrices (fp16) and row factors handed from the chunk-local
                          // kernel to the chain kernel
   size_t off_wdec;       // [n_k + n_v (+ 2 H_v)][d_model] 16-bit decoded weights of the current layer (0 bytes for bf16 weights)
-  size_t off_hist;       // fused: bf16 [n_requests][C][w-1] conv state each request continues from (current layer)
+  size_t off_hist;       // bf16 [n_requests][C][w-1] conv state each request continues from (current layer)
   size_t off_x16;        // fp16 staging: half [max_slots][64][d_model] anchors of the current layer, slot order
   size_t total;
   int64_t max_slots;
@@ -92,14 +97,13 @@ static inline SrWorkspace sr_workspace_layout(const sr_ctx* ctx, int32_t n_reque
   w.off_slot_rows = at; at = sr_align256(at + sizeof(int32_t) * (size_t)w.max_slots);
   w.off_slot_first = at; at = sr_align256(at + sizeof(int32_t) * (size_t)w.max_slots);
   const size_t n_kv = (size_t)ctx->n_k + ctx->n_v;
-  w.off_kv16 = at;      at = sr_align256(at + (ctx->fused ? sizeof(uint16_t) * (size_t)w.max_slots * SR_PAGE_ROWS * n_kv : 0));
-  w.off_zraw = at;      at = sr_align256(at + (ctx->fused ? sizeof(float) * (size_t)w.max_slots * 6 * n_kv : 0));
-  // the projection scratch: all k | v | gate columns, or (fused) the gate columns only
-  w.off_z = at;         at = sr_align256(at + sizeof(float) * (size_t)w.max_slots * SR_PAGE_ROWS *
-                                                  (size_t)(ctx->fused ? ctx->n_gate : ctx->ldz));
-  w.off_split = at;     at = sr_align256(at + (ctx->fused ? sr_scan_split_bytes(ctx, w.max_slots) : 0));
+  const size_t kv_pitch = (n_kv + 127) / 128 * 128;     // channels per slot in the hand-over tiles (whole 128-channel tiles)
+  w.off_kv16 = at;      at = sr_align256(at + sizeof(uint16_t) * (size_t)w.max_slots * SR_PAGE_ROWS * kv_pitch);
+  w.off_zraw = at;      at = sr_align256(at + sizeof(float) * (size_t)w.max_slots * 6 * n_kv);
+  w.off_z = at;         at = sr_align256(at + sizeof(float) * (size_t)w.max_slots * SR_PAGE_ROWS * (size_t)ctx->n_gate);
+  w.off_split = at;     at = sr_align256(at + sr_scan_split_bytes(ctx, w.max_slots));
   w.off_wdec = at;      at = sr_align256(at + ctx->wdec_bytes);
-  w.off_hist = at;      at = sr_align256(at + (ctx->fused ? sizeof(uint16_t) * (size_t)n_requests * ctx->conv_ch * (SR_CONV_W - 1) : 0));
+  w.off_hist = at;      at = sr_align256(at + sizeof(uint16_t) * (size_t)n_requests * ctx->conv_ch * (SR_CONV_W - 1));
   w.off_x16 = at;       at = sr_align256(at + (ctx->fp16_stage ? sizeof(uint16_t) * (size_t)w.max_slots * SR_PAGE_ROWS *
                                                                      (size_t)ctx->desc.d_model : 0));
   w.total = at;
@@ -138,22 +142,23 @@ static inline SrSched sr_sched_view(void* workspace, const SrWorkspace& w, int32
   return s;
 }
 
-// The fused intermediate format between the projection epilogue and the chunk scan (d_k = d_v = 128).
-// Tiles are channel-major: one 128-channel block (a head's k or v) of one 64-row page slot is
-// [128 channels][64 rows], 16 KB, contiguous.
+// The fused intermediate format between the projection epilogue and the chunk scan.  Tiles are channel-major:
+// the k | v channels of one 64-row page slot are [ncb * 128 channels][64 rows] (the channel count rounded up to
+// whole 128-channel projection tiles), so a head's keys (d_k channels) or values (d_v channels) of one slot
+// are one contiguous [channels][64 rows] block.
 struct SrFused {
   const __nv_bfloat16* hist;  // conv state the requests continue from, [request][C][w-1] (current layer), or null = zero
   const char* in_ssm_layer;   // recurrent states the requests continue from (current layer; slot stride below), or null
   int64_t in_ssm_slot_stride;
   const __half* x16; // fp16 staging only: the layer's anchors in slot order [slot][64][d_model], else null
   const __half* w16; // fp16 staging only: dequantised k | v weight rows, then the 2 H_v gate rows, [.][d_model]
-  __half* kv16;      // [slot][column block][128][64] = SiLU(conv(Z)) in fp16.  Rows 0..2 of a slot whose conv
+  __half* kv16;      // [slot][ncb * 128][64] = SiLU(conv(Z)) in fp16.  Rows 0..2 of a slot whose conv
                      // history lies in another projection tile (slot % fix_mod == 0 and not the first slot of
                      // its request) are placeholders: the scan recomputes them from zraw
   float* zraw;       // [slot][6][n_kv] raw fp32 projection rows: 0,1,2 (slots with slot % fix_mod == 0) |
                      // the slot's last three valid rows (every slot)
   float* gates;      // [slot][2 H_v][64] raw fp32 gate pre-activations: a_0.., b_0.. (channel-major)
-  int32_t ncb;       // column blocks: (n_k + n_v) / 128
+  int32_t ncb;       // 128-channel blocks per slot: ceil((n_k + n_v) / 128)
   int32_t n_kv;
   int32_t n_gate;
   int32_t fix_mod;   // page slots per projection tile along the token axis
@@ -170,22 +175,15 @@ struct SrPoolView {
 // Packs the batch: validates each request on the device, assigns page slots, fills the tables.
 cudaError_t sr_launch_schedule(const SrSched& s, const int32_t* pages, const int32_t* state_slots,
                                const int32_t* replay_lens, int32_t max_pages, int32_t max_replay_len,
-                               int64_t max_total_rows, int32_t n_phys_pages, cudaStream_t stream);
+                               int64_t max_total_rows, int32_t n_phys_pages, int32_t n_state_slots,
+                               cudaStream_t stream);
 
 // Copies the gathered rows of one pool layer into a packed [rows][d_model] bf16 array.
 cudaError_t sr_launch_debug_gather(const SrSched& s, const SrPoolView& pool, int32_t pool_layer,
                                    int32_t d_model, int32_t max_pages, void* out_rows,
                                    int64_t out_capacity_rows, cudaStream_t stream);
 
-// Z[slot*64 + r][0 .. n_z) = anchors(slot, r) . W^T for the k | v | a | b columns (CUDA-core version).
-cudaError_t sr_launch_proj_simt(const sr_ctx* ctx, const SrSched& s, const SrPoolView& pool, int32_t pool_layer,
-                                const sr_layer_weights& w, float* z, cudaStream_t stream);
-
-// The same projection on tcgen05 tensor cores with TMA-gathered operands (bf16 weights).
-// For e4m3 weights the codes are first decoded (exactly) to bf16 into `decoded`, a workspace buffer of
-// sr_proj_umma_decoded_bytes, and the block scales are applied to per-128-deep partial sums in fp32.
-bool sr_proj_umma_supported(const sr_ctx* ctx);
-size_t sr_proj_umma_decoded_bytes(const sr_ctx* ctx);
+// block-scaled weights, exact form: the bare e4m3 codes of the k | v rows decoded (exactly) to bf16 into `decoded`
 cudaError_t sr_launch_weight_decode(const sr_ctx* ctx, const sr_layer_weights& w, void* decoded, cudaStream_t stream);
 // continuation: copies the layer's conv states of the batch from the caller's array (by state slot) into the
 // workspace (by request), so that the kernels never read an array the same call writes (sr_conv_tail.cu)
@@ -200,14 +198,12 @@ cudaError_t sr_launch_anchor_write(const sr_anchor_pool& pool, const int32_t* po
 cudaError_t sr_launch_stage_weights_fp16(const sr_ctx* ctx, const sr_layer_weights& w, __half* w16, cudaStream_t stream);
 cudaError_t sr_launch_stage_anchors_fp16(const sr_ctx* ctx, const SrSched& s, const SrPoolView& pool, int32_t pool_layer,
                                          __half* x16, cudaStream_t stream);
-cudaError_t sr_launch_proj_umma(const sr_ctx* ctx, const SrSched& s, const sr_anchor_pool& pool, int32_t pool_layer,
-                                const sr_layer_weights& w, const void* decoded, float* z, int sm_count,
-                                cudaStream_t stream);
 
 // The projection with channels on the MMA's M axis and tokens on its N axis, so that each epilogue
 // thread owns one channel and walks its tokens in order: the causal conv and SiLU are applied in
 // registers and the fused format (SrFused) is written instead of fp32 columns.
 bool sr_proj_fused_supported(const sr_ctx* ctx);
+bool sr_proj_fused_exact_fp8_supported(const sr_ctx* ctx);
 cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_anchor_pool& pool, int32_t pool_layer,
                                  const sr_layer_weights& w, const void* decoded, const SrFused& fused, int sm_count,
                                  cudaStream_t stream);
@@ -215,25 +211,15 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
 // Conv state: last w-1 projection rows of every channel, rounded to bf16.
 int sr_conv_tail_launches(const sr_ctx* ctx);
 cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoolView& pool, int32_t pool_layer,
-                                const sr_layer_weights& w, const float* z, const SrFused* fused, char* out_conv_layer,
+                                const sr_layer_weights& w, const SrFused& fused, char* out_conv_layer,
                                 int64_t slot_stride, cudaStream_t stream);
-
-// conv + SiLU + key norm + gates + token-by-token gated delta rule, one block per (head, request).
-bool sr_scan_token_supported(int d_k, int d_v);
-cudaError_t sr_launch_scan_token(const sr_ctx* ctx, const SrSched& s, const sr_layer_weights& w, const float* z,
-                                 char* out_ssm_layer, int64_t slot_stride, cudaStream_t stream);
 
 // The chunked scan in two kernels for the fused format: everything local to a chunk (gates, K K^T, the
 // inverse) for all chunks at once, then the state chain per (head, request).
+bool sr_chunk_local_supported(int d_k, int d_v);
 cudaError_t sr_launch_chunk_local(const sr_ctx* ctx, const SrSched& s, const sr_layer_weights& w, const SrFused& fused,
                                   void* split_buf, cudaStream_t stream);
-cudaError_t sr_launch_scan_chain(const sr_ctx* ctx, const SrSched& s, const SrFused& fused, const void* split_buf,
-                                 char* out_ssm_layer, int64_t slot_stride, cudaStream_t stream);
-// The same chain on tcgen05 tensor cores with the state in tensor memory.
+// (tcgen05 tensor cores, the state in tensor memory)
+bool sr_scan_chain_supported(int d_k, int d_v);
 cudaError_t sr_launch_scan_chain_umma(const sr_ctx* ctx, const SrSched& s, const SrFused& fused, const void* split_buf,
-                                      char* out_ssm_layer, int64_t slot_stride, cudaStream_t stream);
-
-// The same scan 64 rows at a time on tensor cores (d_k = d_v = 128).
-bool sr_scan_chunk_supported(const sr_ctx* ctx);
-cudaError_t sr_launch_scan_chunk(const sr_ctx* ctx, const SrSched& s, const sr_layer_weights& w, const float* z,
-                                 char* out_ssm_layer, int64_t slot_stride, cudaStream_t stream);
+                                      char* out_ssm_layer, int64_t slot_stride, int sm_count, cudaStream_t stream);

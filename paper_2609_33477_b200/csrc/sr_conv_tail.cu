@@ -3,11 +3,13 @@
 //
 //   out_conv[slot][c][j] = bf16( Z[R - (w-1) + j][c] ),  j = 0 .. w-2, zero for rows before the window
 //
-// The k and v channels are read from the projection scratch.  The q channels are the only use the
+// The k and v channels are read from the raw rows the projection kept.  The q channels are the only use the
 // path has for the query projection, so they are computed here, for the last w-1 rows of each
-// request only.  With bf16 weights that is one skinny GEMM over the whole batch -- (w-1) B gathered anchor
-// rows x n_q channels -- on mma.sync tiles (sr_conv_tail_q_kernel), so every weight row is read once per 64
-// rows instead of once per request; block-scaled weights keep plain dot products, one warp per channel.
+// request only: one skinny GEMM over the whole batch -- (w-1) B gathered anchor rows x channels -- on mma.sync
+// tiles (sr_conv_tail_gemm_kernel), so every weight row is read once per 64 rows instead of once per request.
+// With block-scaled weights that GEMM covers the k and v channels too (codes and scales in fp32), because the
+// projection's copies of those rows went through a rounded 16-bit weight.  Plain dot products, one warp per
+// channel, serve the geometries the tiles do not divide.
 #include "sr_mma.cuh"
 
 namespace {
@@ -20,8 +22,8 @@ __device__ __forceinline__ float e4m3_to_float(uint8_t code) {
 template <bool FP8>
 __global__ void __launch_bounds__(256)
 sr_conv_tail_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_model, int32_t n_q, int32_t c_begin, int32_t conv_ch,
-                    int32_t ldz, const void* __restrict__ w_qkv, const float* __restrict__ w_scale,
-                    const float* __restrict__ z, const float* __restrict__ zraw, int32_t n_kv,
+                    const void* __restrict__ w_qkv, const float* __restrict__ w_scale,
+                    const float* __restrict__ zraw, int32_t n_kv,
                     const __nv_bfloat16* __restrict__ hist, char* __restrict__ out_layer, int64_t slot_stride) {
   const int i = blockIdx.y;
   const int out_slot = s.req_out[i];
@@ -39,13 +41,11 @@ sr_conv_tail_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_mo
     if (lane < SR_CONV_W - 1) {
       const int t = R - (SR_CONV_W - 1) + lane;
       float v = 0.f;
-      if (t >= 0 && zraw) {
-        // fused format: the projection kept the last three valid raw rows of every slot
+      if (t >= 0) {
+        // the projection kept the last three valid raw rows of every slot
         const int slot = slot0 + t / SR_PAGE_ROWS, rho = t % SR_PAGE_ROWS;
         const int idx = 3 + rho - max(s.slot_rows[slot] - 3, 0);
         v = zraw[((int64_t)slot * 6 + idx) * n_kv + (c - n_q)];
-      } else if (t >= 0) {
-        v = z[((int64_t)slot0 * SR_PAGE_ROWS + t) * ldz + (c - n_q)];
       }
       val[0] = v;   // lane j holds entry j
     }
@@ -108,17 +108,23 @@ sr_conv_tail_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_mo
   }
 }
 
-// q channels, bf16 weights: out[r][c] = sum_k X[r][k] W[c][k] for the gathered tail rows r = 3 i + j (request
-// i, window entry j).  One CTA = 64 rows x 64 channels, four warps of 16 rows each, k in chunks of 64 through a
-// two-stage cp.async ring.  Rows without a source (before a request's first token, past the batch, skipped
-// requests) read some valid row and are masked on output.
+// Channels as one GEMM over the batch: out[r][c] = sum_k X[r][k] W[c][k] for the gathered tail rows r = 3 i + j
+// (request i, window entry j).  One CTA = 64 rows x 64 channels, four warps of 16 rows each, k in chunks of 64 through
+// a two-stage ring (cp.async for the anchor rows and for bf16 weights).  Rows without a source (before a request's
+// first token, past the batch, skipped requests) read some valid row and are masked on output.
+//   FP8 = false: bf16 weights, the q channels only (k, v rows come from the projection).
+//   FP8 = true : e4m3 codes with 128 x 128 block scales, every channel q | k | v.  The bare codes are decoded to
+//                bf16 (exact) on their way into shared memory, every 128-deep k group is summed on its own and
+//                enters the result as scale x partial sum in fp32 -- the weights are never rounded, so the conv
+//                state of block-scaled layers is as exact as the one of bf16 layers.
 constexpr int QT = 64;            // tile rows, tile channels and k chunk
 constexpr int QLD = QT + 8;       // shared-memory pitch (bf16)
 
+template <bool FP8>
 __global__ void __launch_bounds__(128)
-sr_conv_tail_q_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_model, int32_t conv_ch,
-                      const __nv_bfloat16* __restrict__ w_q, const __nv_bfloat16* __restrict__ hist,
-                      char* __restrict__ out_layer, int64_t slot_stride) {
+sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_model, int32_t conv_ch,
+                         const void* __restrict__ w_rows, const float* __restrict__ w_scale,
+                         const __nv_bfloat16* __restrict__ hist, char* __restrict__ out_layer, int64_t slot_stride) {
   __shared__ __align__(16) __half Xs[2][QT * QLD];
   __shared__ __align__(16) __half Ws[2][QT * QLD];
   const int tid = threadIdx.x, warp = tid >> 5, l = tid & 31, g8 = l >> 2, t4 = l & 3;
@@ -140,28 +146,49 @@ sr_conv_tail_q_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_
       }
     }
     xrow[q] = src + seg * 16;
-    wrow[q] = (const char*)(w_q + (int64_t)(c0 + m) * d_model) + seg * 16;
+    // bf16: 16 bytes = 8 weights per thread and row; e4m3: 8 bytes = 8 codes
+    wrow[q] = (const char*)w_rows + ((int64_t)(c0 + m) * d_model + seg * 8) * (FP8 ? 1 : 2);
   }
+  uint2 wcode[4];                  // FP8: the next chunk's codes, in registers until their buffer is free
+  auto fetch_codes = [&](int kc) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) wcode[q] = __ldg((const uint2*)(wrow[q] + (int64_t)kc * QT));
+  };
+  auto store_codes = [&](int b) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int m = (tid >> 3) + 16 * q;
+      const uint8_t* e = (const uint8_t*)&wcode[q];
+      __align__(16) __nv_bfloat16 o[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) o[k] = __float2bfloat16_rn(e4m3_to_float(e[k]));   // exact: 4 significant bits
+      *(uint4*)(Ws[b] + m * QLD + seg * 8) = *(const uint4*)o;
+    }
+  };
   auto load = [&](int kc, int b) {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int m = (tid >> 3) + 16 * q;
       cp_async16(Xs[b] + m * QLD + seg * 8, xrow[q] + (int64_t)kc * QT * 2);
-      cp_async16(Ws[b] + m * QLD + seg * 8, wrow[q] + (int64_t)kc * QT * 2);
+      if (!FP8) cp_async16(Ws[b] + m * QLD + seg * 8, wrow[q] + (int64_t)kc * QT * 2);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  float acc[8][4];
+  float acc[8][4], total[8][4];
 #pragma unroll
   for (int n = 0; n < 8; ++n)
 #pragma unroll
-    for (int c = 0; c < 4; ++c) acc[n][c] = 0.f;
+    for (int c = 0; c < 4; ++c) { acc[n][c] = 0.f; total[n][c] = 0.f; }
   const int nk = d_model / QT;
+  const float* scale_row = FP8 ? w_scale + (int64_t)(c0 / 128) * (d_model / 128) : nullptr;
   load(0, 0);
+  if (FP8) fetch_codes(0);
   for (int kc = 0; kc < nk; ++kc) {
     const int b = kc & 1;
+    if (FP8) store_codes(b);       // buffer b was last read two chunks ago; a barrier closed that chunk
     if (kc + 1 < nk) {
       load(kc + 1, b ^ 1);
+      if (FP8) fetch_codes(kc + 1);
       asm volatile("cp.async.wait_group 1;" ::: "memory");
     } else {
       asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -179,6 +206,13 @@ sr_conv_tail_q_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_
       }
     }
     __syncthreads();
+    if (FP8 && (kc & 1)) {         // a 128-deep k group is complete: it shares one block scale
+      const float sc = __ldg(scale_row + (kc >> 1));
+#pragma unroll
+      for (int n = 0; n < 8; ++n)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) { total[n][c] = fmaf(sc, acc[n][c], total[n][c]); acc[n][c] = 0.f; }
+    }
   }
 #pragma unroll
   for (int hr = 0; hr < 2; ++hr) {
@@ -193,7 +227,8 @@ sr_conv_tail_q_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
       const int c = c0 + n * 8 + 2 * t4;
-      __nv_bfloat16 o0 = __float2bfloat16_rn(t >= 0 ? acc[n][2 * hr] : 0.f), o1 = __float2bfloat16_rn(t >= 0 ? acc[n][2 * hr + 1] : 0.f);
+      const float v0 = FP8 ? total[n][2 * hr] : acc[n][2 * hr], v1 = FP8 ? total[n][2 * hr + 1] : acc[n][2 * hr + 1];
+      __nv_bfloat16 o0 = __float2bfloat16_rn(t >= 0 ? v0 : 0.f), o1 = __float2bfloat16_rn(t >= 0 ? v1 : 0.f);
       if (old) {
         o0 = old[(int64_t)c * (SR_CONV_W - 1)];
         o1 = old[(int64_t)(c + 1) * (SR_CONV_W - 1)];
@@ -245,48 +280,54 @@ sr_hist_gather_kernel(SrSched s, const char* __restrict__ in_layer, int64_t slot
 
 }  // namespace
 
-// kernels one sr_launch_conv_tail call launches: the batched q GEMM plus the k | v copy, or the single dot-product kernel
+// kernels one sr_launch_conv_tail call launches: bf16 weights, the batched q GEMM plus the k | v copy; block-scaled
+// weights, one GEMM over all channels; geometries the 64-wide tiles do not divide, the single dot-product kernel
+static bool conv_tail_gemm_fits(const sr_ctx* ctx) {
+  const bool fp8 = ctx->desc.weight_format == SR_W_E4M3_BLOCK128;
+  return (fp8 ? ctx->conv_ch : ctx->n_k) % QT == 0 && ctx->desc.d_model % (fp8 ? 128 : QT) == 0 &&
+         !(ctx->debug_flags & SR_DEBUG_DOT_CONV_STATE);
+}
+
 int sr_conv_tail_launches(const sr_ctx* ctx) {
-  const bool gemm = ctx->desc.weight_format != SR_W_E4M3_BLOCK128 && ctx->n_k % QT == 0 && ctx->desc.d_model % QT == 0 &&
-                    !getenv("SR_SIMT_CONV_TAIL");
-  return gemm ? 2 : 1;
+  if (!conv_tail_gemm_fits(ctx)) return 1;
+  return ctx->desc.weight_format == SR_W_E4M3_BLOCK128 ? 1 : 2;
 }
 
 cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoolView& pool, int32_t pool_layer,
-                                const sr_layer_weights& w, const float* z, const SrFused* fused, char* out_conv_layer,
+                                const sr_layer_weights& w, const SrFused& fused, char* out_conv_layer,
                                 int64_t slot_stride, cudaStream_t stream) {
-  const float* zraw = fused ? fused->zraw : nullptr;
-  const __nv_bfloat16* hist = fused ? fused->hist : nullptr;
+  const float* zraw = fused.zraw;
+  const __nv_bfloat16* hist = fused.hist;
   const int n_kv = ctx->n_k + ctx->n_v;
+  const int tail_rows = s.n_requests * (SR_CONV_W - 1);
   if (ctx->desc.weight_format == SR_W_E4M3_BLOCK128) {
+    // every channel from codes and scales in fp32: the conv state never sees a rounded weight
+    if (conv_tail_gemm_fits(ctx)) {
+      dim3 g((unsigned)(ctx->conv_ch / QT), (unsigned)((tail_rows + QT - 1) / QT));
+      sr_conv_tail_gemm_kernel<true><<<g, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
+                                                            w.w_qkv_scale, hist, out_conv_layer, slot_stride);
+      return cudaGetLastError();
+    }
     dim3 grid((unsigned)((ctx->conv_ch + 7) / 8), (unsigned)s.n_requests);
-    sr_conv_tail_kernel<true><<<grid, 256, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->n_k, 0,
-                                                        ctx->conv_ch, ctx->ldz, w.w_qkv, w.w_qkv_scale, z, zraw,
-                                                        n_kv, hist, out_conv_layer, slot_stride);
+    sr_conv_tail_kernel<true><<<grid, 256, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, 0,
+                                                        ctx->conv_ch, w.w_qkv, w.w_qkv_scale, zraw, n_kv, hist,
+                                                        out_conv_layer, slot_stride);
     return cudaGetLastError();
   }
-  // bf16 weights: the q channels as one batched GEMM, the k and v channels copied from the projection scratch
+  // bf16 weights: the q channels as one batched GEMM (or by dot products), the k and v channels copied from the
+  // raw rows the projection kept
   const int n_q = ctx->n_k;
-  if (sr_conv_tail_launches(ctx) == 2) {
-    const int tail_rows = s.n_requests * (SR_CONV_W - 1);
+  if (conv_tail_gemm_fits(ctx)) {
     dim3 gq((unsigned)(n_q / QT), (unsigned)((tail_rows + QT - 1) / QT));
-    sr_conv_tail_q_kernel<<<gq, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch,
-                                                  (const __nv_bfloat16*)w.w_qkv, hist, out_conv_layer, slot_stride);
-    if (zraw) {
-      dim3 gkv((unsigned)((n_kv + 255) / 256), (unsigned)s.n_requests);
-      sr_conv_tail_kv_kernel<<<gkv, 256, 0, stream>>>(s, n_q, ctx->conv_ch, zraw, n_kv, hist, out_conv_layer, slot_stride);
-    } else {
-      dim3 gkv((unsigned)((n_kv + 7) / 8), (unsigned)s.n_requests);
-      sr_conv_tail_kernel<false><<<gkv, 256, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, n_q, n_q, ctx->conv_ch,
-                                                           ctx->ldz, w.w_qkv, nullptr, z, zraw, n_kv, hist,
-                                                           out_conv_layer, slot_stride);
-    }
+    sr_conv_tail_gemm_kernel<false><<<gq, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
+                                                             nullptr, hist, out_conv_layer, slot_stride);
+    dim3 gkv((unsigned)((n_kv + 255) / 256), (unsigned)s.n_requests);
+    sr_conv_tail_kv_kernel<<<gkv, 256, 0, stream>>>(s, n_q, ctx->conv_ch, zraw, n_kv, hist, out_conv_layer, slot_stride);
     return cudaGetLastError();
   }
   dim3 grid((unsigned)((ctx->conv_ch + 7) / 8), (unsigned)s.n_requests);
   sr_conv_tail_kernel<false><<<grid, 256, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, n_q, 0, ctx->conv_ch,
-                                                       ctx->ldz, w.w_qkv, nullptr, z, zraw, n_kv, hist, out_conv_layer,
-                                                       slot_stride);
+                                                       w.w_qkv, nullptr, zraw, n_kv, hist, out_conv_layer, slot_stride);
   return cudaGetLastError();
 }
 

@@ -1,4 +1,5 @@
-// fp16 staging for e4m3 weights with 128 x 128 block scales (W8A16, Section 7.1 precision setting).
+// Operand staging for e4m3 weights with 128 x 128 block scales (W8A16, Section 7.1 precision setting): the fp16
+// copies the default projection multiplies, and the exact bf16 decode of the bare codes for the fp32-promotion form.
 //
 // The tensor cores take both operands of one product in the same 16-bit format.  Rounding code x scale to bf16
 // (8 significant bits) would cost about 1e-3 relative error per projected value, too close to the state
@@ -45,6 +46,23 @@ sr_stage_weights_fp16_kernel(const uint8_t* __restrict__ codes, const float* __r
   *(uint4*)(out + e0 + 8) = *(const uint4*)(o + 8);
 }
 
+// e4m3 codes -> the same values in bf16 (exact: 4 significant bits fit in 8), no scale applied
+__global__ void __launch_bounds__(256)
+sr_decode_e4m3_kernel(const uint8_t* __restrict__ codes, __nv_bfloat16* __restrict__ out, long long n16) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;     // 16 codes per thread
+  if (i >= n16) return;
+  const uint4 v = *(const uint4*)(codes + i * 16);
+  const uint8_t* e = (const uint8_t*)&v;
+  __align__(16) __nv_bfloat16 o[16];
+#pragma unroll
+  for (int q = 0; q < 16; ++q) {
+    const __half_raw hr = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)e[q], __NV_E4M3);
+    o[q] = __float2bfloat16_rn(__half2float(__half(hr)));
+  }
+  *(uint4*)(out + i * 16) = *(const uint4*)o;
+  *(uint4*)(out + i * 16 + 8) = *(const uint4*)(o + 8);
+}
+
 // one CTA per page slot: 64 rows x d_model, 8 values per thread and step
 __global__ void __launch_bounds__(256)
 sr_stage_anchors_fp16_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_model, __half* __restrict__ x16) {
@@ -83,6 +101,15 @@ cudaError_t sr_launch_stage_weights_fp16(const sr_ctx* ctx, const sr_layer_weigh
   const uint8_t* src = (const uint8_t*)w.w_qkv + (long long)ctx->n_k * d;      // the q rows are skipped
   sr_stage_weights_fp16_kernel<<<(unsigned)((n16_all + 255) / 256), 256, 0, stream>>>(
       src, w.w_qkv_scale, (const __nv_bfloat16*)w.w_ab, w16, n16_kv, n16_all, d, ctx->n_k);
+  return cudaGetLastError();
+}
+
+cudaError_t sr_launch_weight_decode(const sr_ctx* ctx, const sr_layer_weights& w, void* decoded, cudaStream_t stream) {
+  // the k | v rows of the e4m3 code matrix (the q rows are skipped), 16 codes per thread
+  const long long n = (long long)(ctx->n_k + ctx->n_v) * ctx->desc.d_model;
+  const uint8_t* src = (const uint8_t*)w.w_qkv + (long long)ctx->n_k * ctx->desc.d_model;
+  const long long n16 = n / 16;
+  sr_decode_e4m3_kernel<<<(unsigned)((n16 + 255) / 256), 256, 0, stream>>>(src, (__nv_bfloat16*)decoded, n16);
   return cudaGetLastError();
 }
 

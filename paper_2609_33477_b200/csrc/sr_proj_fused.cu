@@ -20,8 +20,6 @@
 // 128 x 128 block scales: 128-deep K groups are accumulated separately and added as scale x partial sum in
 // fp32 registers by eight epilogue warps (one scale per K group per tile, since a tile is one 128-channel
 // block).  All waits are bounded.
-#include <stdlib.h>
-
 #include "sr_umma.cuh"
 
 namespace {
@@ -70,8 +68,17 @@ __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
 // One page slot (64 tokens, in v) of one channel: conv + SiLU -> fp16 tile row, raw rows -> zraw;
 // or, for the gate tile, the raw values -> gates.  z1, z2, z3 carry the three previous raw tokens.
 __device__ __forceinline__ void emit_slot(const FusedParams& p, bool gate, int ch, int ch_local, int ct, int slot,
-                                          bool head_rows, int vr, const float* v, const float (&cw)[4], float& z1,
+                                          bool head_rows, int vr, float* v, const float (&cw)[4], float& z1,
                                           float& z2, float& z3) {
+  // Rows past the request's end (a partial last page, a padding slot) are not part of the window: whatever the
+  // pool holds there -- stale anchors, never-written memory, NaN -- must not reach the scan, whose products mix
+  // the rows of a chunk.  vr is uniform over the warp.
+  if (vr < SR_PAGE_ROWS) {
+#pragma unroll
+    for (int i = 0; i < SR_PAGE_ROWS; ++i)
+      if (i >= vr) v[i] = 0.f;
+  }
+  if (!gate && ch >= p.n_kv) return;     // the last channel tile may reach past the k | v block
   if (gate) {
     if (ch < p.n_gate) {
       float* g = p.gates + ((long long)slot * p.n_gate + ch) * SR_PAGE_ROWS;
@@ -120,7 +127,7 @@ __device__ __forceinline__ void emit_slot(const FusedParams& p, bool gate, int c
 __device__ __forceinline__ void load_history(const FusedParams& p, bool gate, int first, int ch, float& z1, float& z2,
                                              float& z3) {
   z1 = 0.f; z2 = 0.f; z3 = 0.f;
-  if (first && p.hist && !gate) {
+  if (first && p.hist && !gate && ch < p.n_kv) {
     const __nv_bfloat16* h = p.hist + ((long long)(first - 1) * p.conv_ch + p.n_q + ch) * (SR_CONV_W - 1);
     z3 = __bfloat162float(h[0]);
     z2 = __bfloat162float(h[1]);
@@ -251,7 +258,7 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       const bool gate = ct == p.n_ct;
       const int ch = gate ? ch_local : ct * BM + ch_local;
       float cw[4] = {0.f, 0.f, 0.f, 0.f};
-      if (!gate) {
+      if (!gate && ch < p.n_kv) {
         const uint2 wv = *(const uint2*)(p.conv_w + (long long)(p.n_q + ch) * SR_CONV_W);
         const __nv_bfloat16* e = (const __nv_bfloat16*)&wv;
 #pragma unroll
@@ -350,7 +357,8 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int n_slots = (int)p.s.status[1];
   const int t_tiles = (n_slots + SLOTS - 1) / SLOTS;
-  const int n_pt = p.n_ct / 2;                    // 256-channel tiles of k | v; tile index n_pt is the gate tile
+  const int n_pt = (p.n_ct + 1) / 2;              // 256-channel tiles of k | v (the last may be half empty); tile
+                                                  // index n_pt is the gate tile
   const int c_tiles = n_pt + 1;
   const long long total_tiles = (long long)t_tiles * c_tiles;
 
@@ -450,7 +458,7 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
       const int ct = 2 * pt + rank;                       // this CTA's 128-channel block
       const int ch = gate ? rank * BM + ch_local : ct * BM + ch_local;
       float cw[4] = {0.f, 0.f, 0.f, 0.f};
-      if (!gate) {
+      if (!gate && ch < p.n_kv) {
         const uint2 wv = *(const uint2*)(p.conv_w + (long long)(p.n_q + ch) * SR_CONV_W);
         const __nv_bfloat16* e = (const __nv_bfloat16*)&wv;
 #pragma unroll
@@ -488,10 +496,15 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
 }  // namespace
 
 bool sr_proj_fused_supported(const sr_ctx* ctx) {
-  if (ctx->desc.d_k != 128 || ctx->desc.d_v != 128) return false;
-  if (ctx->desc.d_model % BK != 0 || ctx->n_gate > BM) return false;
+  // any head geometry: the projection works on channels, in tiles of 128 (the last one may be partial)
+  if (ctx->desc.d_model % BK != 0 || ctx->n_gate > 2 * BM) return false;
   if (ctx->desc.weight_format == SR_W_E4M3_BLOCK128) return ctx->desc.d_model % 128 == 0;
   return true;
+}
+
+// fp32 promotion of bare-code partial sums needs every 128-channel tile inside one row block of the scales
+bool sr_proj_fused_exact_fp8_supported(const sr_ctx* ctx) {
+  return ctx->n_k % BM == 0 && (ctx->n_k + ctx->n_v) % BM == 0 && ctx->n_gate <= BM;
 }
 
 cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_anchor_pool& pool, int32_t pool_layer,
@@ -537,7 +550,7 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   p.k_blocks = d / BK;
   p.n_q = ctx->n_k;
   p.w_row0 = (scaled || stage) ? 0 : ctx->n_k;
-  p.n_ct = n_kv / BM;
+  p.n_ct = (n_kv + BM - 1) / BM;
   p.n_gate = ctx->n_gate;
   p.ncb = fused.ncb;
   p.n_kv = n_kv;
@@ -549,40 +562,35 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   p.zraw = fused.zraw;
   p.gates = fused.gates;
 
-  static bool attr_set = false;
-  if (!attr_set) {
+  cudaError_t once = sr_once_per_device(SR_ONCE_PROJ_FUSED, [] {
     cudaError_t e = cudaFuncSetAttribute(sr_proj_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(sr_proj_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+    return e;
+  });
+  if (once != cudaSuccess) return once;
   const long long max_tiles = (long long)(s.max_slots / SLOTS) * (p.n_ct + 1);
   int grid = (int)(max_tiles < sm_count ? max_tiles : sm_count);
   if (grid < 1) grid = 1;
-  const char* one = getenv("SR_SINGLE_CTA_MMA");
-  const bool pair_form = !scaled && p.n_ct % 2 == 0 && sm_count >= 2 && !(one && one[0] == '1');
+  // CTA pairs by default; the one-CTA form serves the exact block-scaled path and (on request) the tests
+  const bool pair_form = !scaled && sm_count >= 2 && (!(ctx->debug_flags & SR_DEBUG_SINGLE_CTA_MMA) || ctx->n_gate > BM);
   // Tile order: the channel tiles are cut into equal blocks of about WEIGHT_BLOCK_BYTES of weights; a block
   // stays in L2 while every token tile streams past it once (channel-fastest inside a block), so weights are
   // read from HBM once and anchors once per block.  Holding anchors instead and streaming the weights past
   // them costs more: measured 17.7 ms against 15.9 ms per launch at 254 400 tokens, d = 5120.
   {
-    const long long c_tiles = pair_form ? p.n_ct / 2 + 1 : p.n_ct + 1;
+    const long long c_tiles = pair_form ? (p.n_ct + 1) / 2 + 1 : p.n_ct + 1;
     const long long tile_bytes = (long long)(pair_form ? 2 * BM : BM) * d * 2;
     const long long blocks = (c_tiles * tile_bytes + WEIGHT_BLOCK_BYTES - 1) / WEIGHT_BLOCK_BYTES;
     p.group_c = (int32_t)((c_tiles + blocks - 1) / blocks);
     p.group_t = 1 << 30;
   }
-  if (const char* e = getenv("SR_GROUP_T")) { const int v = atoi(e); if (v > 0) p.group_t = v; }
-  if (const char* e = getenv("SR_GROUP_C")) { const int v = atoi(e); if (v > 0) p.group_c = v; }
   if (pair_form) {
-    static bool attr2_set = false;
-    if (!attr2_set) {
-      cudaError_t e = cudaFuncSetAttribute(sr_proj_fused2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
-      if (e != cudaSuccess) return e;
-      attr2_set = true;
-    }
-    const long long pair_tiles = (long long)(s.max_slots / SLOTS) * (p.n_ct / 2 + 1);
+    once = sr_once_per_device(SR_ONCE_PROJ_FUSED2, [] {
+      return cudaFuncSetAttribute(sr_proj_fused2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
+    });
+    if (once != cudaSuccess) return once;
+    const long long pair_tiles = (long long)(s.max_slots / SLOTS) * ((p.n_ct + 1) / 2 + 1);
     long long pairs = sm_count / 2;
     if (pair_tiles < pairs) pairs = pair_tiles;
     if (pairs < 1) pairs = 1;

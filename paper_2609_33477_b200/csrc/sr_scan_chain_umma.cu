@@ -17,6 +17,12 @@
 //   -W^T       written by the threads from tensor memory as [d_k][64]: an MN-major B operand of S^T W^T
 //   S (fp16)   written by the threads as [d_k][d_v] in two 64-column halves: an MN-major A operand
 //   (f U)^T    written by the threads as [d_v][64]: a K-major B operand of the state update
+// Head widths other than 128: every product keeps M = 128.  Tiles are fetched 128 channels tall whatever d_k and
+// d_v are, so lanes past a head's own channels hold its neighbours' channels (or stale scratch): their results
+// are never read -- the one contraction over the key index, S^T W^T, runs over d_k only, value columns never mix
+// (Eq. 5: the state is linear in the values, column by column), and only rows < d_k, columns < d_v are stored.
+// A value head wider than 128 is split into equal column blocks of at most 128, one CTA each; narrower heads
+// may be split too, to put more CTAs on a small batch.
 // Tensor memory (256 columns per CTA, two CTAs per SM): S fp32 (lanes d_k, 128 columns), U^T (lanes d_v,
 // 64 columns), W^T (lanes d_k, 64 columns).  Eight warps move data between tensor memory and shared memory
 // (warp w works on lanes 32 (w % 4) .. and on one half of the columns); a ninth warp's first lane issues the
@@ -31,7 +37,7 @@
 namespace {
 
 constexpr int CH = 64;
-constexpr int D = 128;
+constexpr int D = 128;                   // tile height and MMA M: head widths up to 128 per CTA
 constexpr int TT_HALFS = 2 * CH * CH;
 constexpr int SC_FLOATS = 128;
 constexpr int COMPUTE_THREADS = 256;
@@ -62,11 +68,16 @@ struct ChainUmmaParams {
   const float* sc;
   int32_t ncb;
   int32_t n_k_heads, n_v_heads;
+  int32_t d_k, d_v;          // head widths
+  int32_t dvb;               // value columns per CTA (d_v / gridDim.z, a multiple of 4, at most 128)
   char* out_layer;
   int64_t slot_stride;
   int32_t erase;             // 0: decay-only family, U = U~ (no W S term)
   const char* in_layer;      // states to continue from (same slot addressing as the output), or null = zero
   int64_t in_slot_stride;
+  long long wait_limit;      // cycles a wait may take before it gives up
+  int32_t withhold_first_keys;   // fault injection (SR_DEBUG_EXPIRE_WAIT): chunk 0's key tile is never requested, so
+                                 // the waits on it run out
 };
 
 // instruction descriptor: D fp32, A and B fp16, M x N, operand majors (0 = K-major, 1 = MN-major)
@@ -128,17 +139,23 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
   if (out_slot < 0) return;
   const int R = p.s.req_rows[req];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  float* out = (float*)(p.out_layer + (int64_t)out_slot * p.slot_stride) + (int64_t)h * D * D;
+  const int dk = p.d_k, dv = p.d_v, dvb = p.dvb, col0 = (int)blockIdx.z * dvb;     // this CTA: value columns col0 .. col0 + dvb
+  const int64_t head_off = (int64_t)h * dk * dv + col0;
+  float* out = (float*)(p.out_layer + (int64_t)out_slot * p.slot_stride) + head_off;
   const int kh = h / (p.n_v_heads / p.n_k_heads);
   const int slot0 = p.s.req_slot0[req];
   const int n_chunks = (R + CH - 1) / CH;
-  const float* init = p.in_layer ? (const float*)(p.in_layer + (int64_t)out_slot * p.in_slot_stride) + (int64_t)h * D * D : nullptr;
+  const float* init = p.in_layer ? (const float*)(p.in_layer + (int64_t)out_slot * p.in_slot_stride) + head_off : nullptr;
   const bool has_init = init != nullptr;
   const bool erase = p.erase != 0;
   if (n_chunks == 0) {                 // nothing to replay: the state is handed through (or zero)
-    if (init != out)
-      for (int i = tid; i < D * D / 4; i += THREADS)
-        ((float4*)out)[i] = has_init ? ((const float4*)init)[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    if (init != out) {
+      const int q4 = dvb / 4;          // float4 pieces per row of this CTA's block
+      for (int i = tid; i < dk * q4; i += THREADS) {
+        const int64_t at = (int64_t)(i / q4) * dv + (i % q4) * 4;
+        *(float4*)(out + at) = has_init ? *(const float4*)(init + at) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
     return;
   }
   if ((smem_u32(smem_raw) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment
@@ -165,13 +182,15 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
   const uint32_t tmem_base = sm.tmem_slot;
   const uint32_t tm_S = tmem_base, tm_U = tmem_base + 128, tm_W = tmem_base + 192;
 
-  // tile rows in the tensor maps: key / value tile of (slot, block) starts at row (slot*ncb + block)*128;
+  // tile rows in the tensor maps: channel c of slot s is row s * (ncb * 128) + c (keys of key head a from
+  // a * d_k, values of value head h from H_k d_k + h * d_v), 128 rows fetched whatever the head width;
   // T matrices of (slot, head) start at row (slot*H_v + head)*128 (Tb), +64 (Tw)
+  const int k_row = kh * dk, v_row = p.n_k_heads * dk + h * dv + col0, slot_rows = p.ncb * D;
   auto load_v = [&](int ck) {          // V^T, Tb, Tw of chunk ck (one buffer)
     const int slot = slot0 + ck;
     uint64_t* bar = &sm.bar_v[ck & 1];
     mbar_expect_tx(bar, TILE_KV + 2 * TILE_T);
-    tma_load_2d(sm.VT, &map_kv, bar, 0, (slot * p.ncb + p.n_k_heads + h) * D);
+    tma_load_2d(sm.VT, &map_kv, bar, 0, slot * slot_rows + v_row);
     tma_load_2d(sm.Tb, &map_tt, bar, 0, (slot * p.n_v_heads + h) * 2 * CH);
     tma_load_2d(sm.Tw, &map_tt, bar, 0, (slot * p.n_v_heads + h) * 2 * CH + CH);
   };
@@ -179,7 +198,7 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
     const int slot = slot0 + ck;
     uint64_t* bar = &sm.bar_k[ck & 1];
     mbar_expect_tx(bar, TILE_KV + SC_BYTES);
-    tma_load_2d(sm.KT[ck & 1], &map_kv, bar, 0, (slot * p.ncb + kh) * D);
+    tma_load_2d(sm.KT[ck & 1], &map_kv, bar, 0, slot * slot_rows + k_row);
     bulk_load(sm.sc[ck & 1], p.sc + ((long long)slot * p.n_v_heads + h) * SC_FLOATS, SC_BYTES, bar);
   };
 
@@ -192,7 +211,7 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
     auto issue_ahead = [&](int ck) -> bool {
       const uint32_t par = (uint32_t)((ck >> 1) & 1);
       const int b = ck & 1;
-      if (!(mbar_wait(&sm.bar_v[b], par, abort_flag, p.s.status) && mbar_wait(&sm.bar_k[b], par, abort_flag, p.s.status)))
+      if (!(mbar_wait(&sm.bar_v[b], par, abort_flag, p.s.status, p.wait_limit) && mbar_wait(&sm.bar_k[b], par, abort_flag, p.s.status, p.wait_limit)))
         return false;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t i64 = idesc_f16(D, CH, 0, 1);     // the T tiles are stored [column][row]: MN-major B operands
@@ -207,7 +226,7 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
       umma_commit(&sm.bar_m1[b]);
       if (ck + 1 < n_chunks) {
         // once these (and everything issued before them) are done, V^T, Tb, Tw and the other key buffer are free
-        if (!mbar_wait(&sm.bar_m1[b], par, abort_flag, p.s.status)) return false;
+        if (!mbar_wait(&sm.bar_m1[b], par, abort_flag, p.s.status, p.wait_limit)) return false;
         load_v(ck + 1);
         if (ck > 0) load_k(ck + 1);
       }
@@ -215,7 +234,7 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
     };
     if (lane == 0) {
       load_v(0);
-      load_k(0);
+      if (!p.withhold_first_keys) load_k(0);
       if (n_chunks > 1) load_k(1);
       ok = issue_ahead(0);
     }
@@ -229,7 +248,8 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
           const uint32_t imn = idesc_f16(D, CH, 1, 1);
           const uint64_t a_s = smem_desc(smem_u32(sm.S16), TILE_KV, 1024), b_w = smem_desc(smem_u32(sm.WU), 16, 1024);
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) umma_bf16(tm_U, a_s + 128 * k, b_w + 128 * k, imn, 1u);       // U^T -= S^T W^T
+          for (int k = 0; k < D / 16; ++k)                                                                // U^T -= S^T W^T,
+            if (16 * k < dk) umma_bf16(tm_U, a_s + 128 * k, b_w + 128 * k, imn, 1u);                      // summed over d_k only
         }
         umma_commit(&sm.bar_m2[b]);
       }
@@ -251,14 +271,17 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
     const int row = quarter * 32 + lane;                                // tensor-memory lane = d_k or d_v index
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     if (has_init) {
-      // the state this request continues: row `row`, this warp's 64 columns, into tensor memory
+      // the state this request continues: row `row`, this warp's 64 columns, into tensor memory (zero outside
+      // the head's own rows and this CTA's columns)
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         float v[32];
-        const float* src = init + (int64_t)row * D + half * 64 + c * 32;
+        const int cbase = half * 64 + c * 32;
+        const float* src = init + (int64_t)row * dv + cbase;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) *(float4*)(v + 4 * q) = *(const float4*)(src + 4 * q);
-        tmem_st32(tm_S + lane_off + (uint32_t)(half * 64 + c * 32), v);
+        for (int q = 0; q < 8; ++q)
+          *(float4*)(v + 4 * q) = (row < dk && cbase + 4 * q < dvb) ? *(const float4*)(src + 4 * q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        tmem_st32(tm_S + lane_off + (uint32_t)cbase, v);
       }
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
@@ -266,10 +289,10 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
       const uint32_t par = (uint32_t)((ck >> 1) & 1);
       const int b = ck & 1;
       const float* sc = sm.sc[b];
-      if (ok) ok = mbar_wait(&sm.bar_k[b], par, abort_flag, p.s.status);     // row factors and gamma_n
+      if (ok) ok = mbar_wait(&sm.bar_k[b], par, abort_flag, p.s.status, p.wait_limit);     // row factors and gamma_n
       if ((ck > 0 || has_init) && ok) {
         // the state left by the previous chunk (or the initial one): fp16 copy for S^T W^T, then decay in place
-        if (ck > 0) ok = mbar_wait(&sm.bar_m3[b ^ 1], (uint32_t)(((ck - 1) >> 1) & 1), abort_flag, p.s.status);
+        if (ck > 0) ok = mbar_wait(&sm.bar_m3[b ^ 1], (uint32_t)(((ck - 1) >> 1) & 1), abort_flag, p.s.status, p.wait_limit);
         if (ok) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const float decay = sc[CH];
@@ -285,7 +308,7 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
           asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         }
         // -W^T: this warp's 32 of the 64 chunk-row columns
-        if (ok && erase) ok = mbar_wait(&sm.bar_m1[b], par, abort_flag, p.s.status);
+        if (ok && erase) ok = mbar_wait(&sm.bar_m1[b], par, abort_flag, p.s.status, p.wait_limit);
         if (ok && erase) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           float v[32];
@@ -298,7 +321,7 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncthreads();                                                 // S1
-      if (ok) ok = mbar_wait(&sm.bar_m2[b], par, abort_flag, p.s.status);
+      if (ok) ok = mbar_wait(&sm.bar_m2[b], par, abort_flag, p.s.status, p.wait_limit);
       if (ok) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         float v[32];
@@ -312,16 +335,18 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
       __syncthreads();                                                 // S2
     }
     // ---------------- the final state ----------------
-    if (ok) ok = mbar_wait(&sm.bar_m3[(n_chunks - 1) & 1], (uint32_t)(((n_chunks - 1) >> 1) & 1), abort_flag, p.s.status);
+    if (ok) ok = mbar_wait(&sm.bar_m3[(n_chunks - 1) & 1], (uint32_t)(((n_chunks - 1) >> 1) & 1), abort_flag, p.s.status, p.wait_limit);
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         float v[32];
-        tmem_ld32(tm_S + lane_off + (uint32_t)(half * 64 + c * 32), v);
-        float* dst = out + (int64_t)row * D + half * 64 + c * 32;
+        const int cbase = half * 64 + c * 32;
+        tmem_ld32(tm_S + lane_off + (uint32_t)cbase, v);
+        float* dst = out + (int64_t)row * dv + cbase;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) *(float4*)(dst + 4 * q) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        for (int q = 0; q < 8; ++q)
+          if (row < dk && cbase + 4 * q < dvb) *(float4*)(dst + 4 * q) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
       }
     }
   }
@@ -349,18 +374,29 @@ bool encode_tiles(CUtensorMap* map, const void* base, uint64_t rows, uint32_t bo
 
 }  // namespace
 
+// Column blocks a value head is split into: as few as keep a block within 128 columns (a multiple of 4, for the
+// vector stores), one more doubling while the chains would otherwise leave most SMs without a CTA.
+int sr_scan_chain_value_blocks(int d_v, long long chains, int sm_count) {
+  int n = (d_v + D - 1) / D;
+  while (d_v % n != 0 || (d_v / n) % 4 != 0) ++n;
+  if (chains * n < sm_count && (d_v / n) % 8 == 0 && d_v / (2 * n) >= 32) n *= 2;
+  return n;
+}
+
+bool sr_scan_chain_supported(int d_k, int d_v) {
+  return d_k % 16 == 0 && d_k >= 16 && d_k <= D && d_v % 4 == 0 && d_v > 0 && d_v <= 8 * D;
+}
+
 cudaError_t sr_launch_scan_chain_umma(const sr_ctx* ctx, const SrSched& s, const SrFused& fused, const void* split_buf,
-                                      char* out_ssm_layer, int64_t slot_stride, cudaStream_t stream) {
+                                      char* out_ssm_layer, int64_t slot_stride, int ctx_sm_count, cudaStream_t stream) {
   // fused.in_ssm_layer: states to continue from (may be the output array itself: every CTA reads its block before
   // it writes it)
   const sr_model_desc& d = ctx->desc;
-  static bool attr_set = false;
   const int smem_bytes = (int)sizeof(Smem);
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(sr_scan_chain_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  const cudaError_t once = sr_once_per_device(SR_ONCE_CHAIN_UMMA, [] {
+    return cudaFuncSetAttribute(sr_scan_chain_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Smem));
+  });
+  if (once != cudaSuccess) return once;
   CUtensorMap map_kv, map_tt;
   if (!encode_tiles(&map_kv, fused.kv16, (uint64_t)s.max_slots * fused.ncb * D, D)) return cudaErrorInvalidValue;
   if (!encode_tiles(&map_tt, split_buf, (uint64_t)s.max_slots * d.n_v_heads * 2 * CH, CH)) return cudaErrorInvalidValue;
@@ -370,12 +406,18 @@ cudaError_t sr_launch_scan_chain_umma(const sr_ctx* ctx, const SrSched& s, const
   p.ncb = fused.ncb;
   p.n_k_heads = d.n_k_heads;
   p.n_v_heads = d.n_v_heads;
+  p.d_k = d.d_k;
+  p.d_v = d.d_v;
+  const int n_vb = sr_scan_chain_value_blocks(d.d_v, (long long)d.n_v_heads * s.n_requests, ctx_sm_count);
+  p.dvb = d.d_v / n_vb;
   p.out_layer = out_ssm_layer;
   p.slot_stride = slot_stride;
   p.erase = d.recurrence == SR_REC_GATED_DELTA;
   p.in_layer = fused.in_ssm_layer;
   p.in_slot_stride = fused.in_ssm_slot_stride;
-  dim3 grid((unsigned)d.n_v_heads, (unsigned)s.n_requests);
+  p.withhold_first_keys = (ctx->debug_flags & SR_DEBUG_EXPIRE_WAIT) ? 1 : 0;
+  p.wait_limit = p.withhold_first_keys ? 2000000ll : WAIT_LIMIT_CYCLES;      // about a millisecond for the injected fault
+  dim3 grid((unsigned)d.n_v_heads, (unsigned)s.n_requests, (unsigned)n_vb);
   sr_scan_chain_umma_kernel<<<grid, THREADS, smem_bytes, stream>>>(map_kv, map_tt, p);
   return cudaGetLastError();
 }

@@ -1,4 +1,4 @@
-// The chunked gated-delta scan (Eq. 4, 64 rows at a time) split in two kernels.
+// The chunked gated-delta scan (Eq. 4, 64 rows at a time) split in two kernels; this file holds the first.
 //
 // With g_i the running sum of log alpha inside a chunk, gamma_i = exp(g_i), n_i = 1/sqrt(|k_i|^2 + eps):
 //
@@ -12,10 +12,10 @@
 // no serial chain, latency hidden by occupancy.  It leaves T diag(beta), T diag(beta gamma n) (fp16, stored
 // transposed: [column][row]) and
 // the row factors exp(g_n - g_j) n_j, gamma_n per chunk, and finishes the first three conv rows of chunks
-// whose conv history the projection could not see.  sr_scan_chain_kernel then walks each (head, request)
-// chain with three tensor-core phases per chunk (W and U~; U; state update), state in registers.
+// whose conv history the projection could not see.  The state chain (sr_scan_chain_umma.cu) then walks each
+// (head, request) chain.
 //
-// Products run on mma.sync m16n8k16, fp16 operands (the 11 significant bits of tf32; bf16's 8 would
+// Products here run on mma.sync m16n8k16, fp16 operands (the 11 significant bits of tf32; bf16's 8 would
 // miss the 2e-3 state tolerance), fp32 accumulation.  Row scalings are folded into T's columns and U's
 // rows in fp32 before the single rounding to fp16, so k and v are rounded exactly once.
 #include "sr_mma.cuh"
@@ -23,11 +23,8 @@
 namespace {
 
 constexpr int CH = 64;            // chunk rows (= page rows)
-constexpr int D = 128;            // d_k = d_v
-constexpr int LDH = D + 8;        // pitch (halfs) of row-major [64][128] fp16 tiles
 constexpr int LDT = CH + 8;       // pitch (halfs) of 64 x 64 fp16 tiles
-constexpr int LDK = CH + 8;       // pitch (halfs) of channel-major [128][64] k, v tiles
-constexpr int THREADS = 256;
+constexpr int LDK = CH + 8;       // pitch (halfs) of channel-major [d_k][64] key tiles
 constexpr int TT_HALFS = 2 * CH * CH;   // per chunk and head: T diag(beta), then T diag(beta gamma n)
 constexpr int SC_FLOATS = 128;          // per chunk and head: 64 row factors, gamma_n, padding
 
@@ -41,9 +38,10 @@ constexpr int LT = 128;           // threads of the chunk-local kernel: small CT
 
 constexpr int LDI = 24;           // pitch (halfs) of the fp16 inverses of the diagonal blocks
 
+template <int DK>
 struct LocalSmem {
   union {                         // the key tile is dead once K K^T sits in registers: A takes its place
-    __half Ks[D * LDK];           // keys of the chunk, channel-major
+    __half Ks[DK * LDK];          // keys of the chunk, channel-major
     struct {
       __half A16[CH * LDT];       // A below the block diagonal, fp16 (operand of the block products)
       __half Dinv[4 * 16 * LDI];  // their inverses (I + A_bb)^-1, fp16, row-major
@@ -59,10 +57,11 @@ struct LocalSmem {
 struct LocalParams {
   SrSched s;
   const float* gates;             // [slot][2 H_v][64]
-  __half* kv16;                   // [slot][ncb][128][64]; rows 0..2 are completed here where needed
+  __half* kv16;                   // [slot][ncb * 128 channels][64]; rows 0..2 are completed here where needed
   const float* zraw;              // [slot][6][n_kv]
   int32_t ncb, n_kv, fix_mod;
   int32_t n_k_heads, n_v_heads;
+  int32_t d_v;                    // value head width (the key head width is the template parameter)
   int32_t act_identity;
   int32_t erase;                  // 0: decay-only family, A = 0 and T = I
   float eps;
@@ -96,22 +95,24 @@ __device__ __forceinline__ void pack_right(const float (&x)[2][4], uint32_t (&b)
   }
 }
 
+template <int DK>
 __global__ void __launch_bounds__(LT, LOCAL_CTAS_PER_SM) sr_chunk_local_kernel(const LocalParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  LocalSmem& sm = *reinterpret_cast<LocalSmem*>(smem_raw);
+  LocalSmem<DK>& sm = *reinterpret_cast<LocalSmem<DK>*>(smem_raw);
   const int h = blockIdx.x, slot = blockIdx.y;
   if (slot >= (int)p.s.status[1]) return;
   const int vr = p.s.slot_rows[slot];
   if (vr == 0) return;                                   // padding slot
   const int tid = threadIdx.x, warp = tid >> 5, l = tid & 31, g8 = l >> 2, t4 = l & 3;
   const int kh = h / (p.n_v_heads / p.n_k_heads);
-  const int n_k = p.n_k_heads * D;
+  const int n_k = p.n_k_heads * DK, dv = p.d_v;
   const bool fix = !p.s.slot_first[slot] && (slot % p.fix_mod) == 0;
-  __half* tk = p.kv16 + ((long long)slot * p.ncb + kh) * (CH * D);
-  __half* tv = p.kv16 + ((long long)slot * p.ncb + p.n_k_heads + h) * (CH * D);
+  const long long slot_ch = (long long)slot * p.ncb * 128;        // first channel row of this slot's tiles
+  __half* tk = p.kv16 + (slot_ch + kh * DK) * CH;
+  __half* tv = p.kv16 + (slot_ch + n_k + h * dv) * CH;
 
   // ---- fetch: the key tile and the two gate rows of this head ----
-  for (int i = tid; i < D * (CH / 8); i += LT) {
+  for (int i = tid; i < DK * (CH / 8); i += LT) {
     const int c = i >> 3, seg = i & 7;
     cp_async16(sm.Ks + c * LDK + seg * 8, tk + c * CH + seg * 8);
   }
@@ -121,17 +122,20 @@ __global__ void __launch_bounds__(LT, LOCAL_CTAS_PER_SM) sr_chunk_local_kernel(c
                p.gates + ((long long)slot * (2 * p.n_v_heads) + (which ? p.n_v_heads + h : h)) * CH + seg * 4);
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
-  // where a fix-up is due: the previous slot's last three raw rows and this slot's rows 0..2 of this thread's two
-  // channels (0..127 k, 128..255 v), fetched while the key tile is in flight
-  float zr[2][6];
+  // where a fix-up is due: the previous slot's last three raw rows and this slot's rows 0..2 of this thread's
+  // channels (the head's d_k key channels, then its d_v value channels), fetched while the key tile is in flight
+  constexpr int FIXQ = 3;         // channels per thread: d_k + d_v <= 3 * 128
+  float zr[FIXQ][6];
   if (fix) {
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
+    for (int q = 0; q < FIXQ; ++q) {
       const int c = tid + q * LT;
-      const int zc = c < D ? kh * D + c : n_k + h * D + (c - D);
+      if (c < DK + dv) {
+        const int zc = c < DK ? kh * DK + c : n_k + h * dv + (c - DK);
 #pragma unroll
-      for (int rr = 0; rr < 6; ++rr)
-        zr[q][rr] = __ldg(p.zraw + ((long long)(rr < 3 ? slot - 1 : slot) * 6 + (rr < 3 ? 3 + rr : rr - 3)) * p.n_kv + zc);
+        for (int rr = 0; rr < 6; ++rr)
+          zr[q][rr] = __ldg(p.zraw + ((long long)(rr < 3 ? slot - 1 : slot) * 6 + (rr < 3 ? 3 + rr : rr - 3)) * p.n_kv + zc);
+      }
     }
   }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -141,21 +145,23 @@ __global__ void __launch_bounds__(LT, LOCAL_CTAS_PER_SM) sr_chunk_local_kernel(c
     // rows 0..2: conv over the raw rows, SiLU, fp16; written back to the tiles for the chain kernel (heads
     // sharing a key head write identical key values)
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
+    for (int q = 0; q < FIXQ; ++q) {
       const int c = tid + q * LT;
-      const int zc = c < D ? kh * D + c : n_k + h * D + (c - D);
-      const uint2 wv = *(const uint2*)(p.conv_w + (long long)(n_k + zc) * SR_CONV_W);
-      const __nv_bfloat16* e = (const __nv_bfloat16*)&wv;
-      const float w0 = __bfloat162float(e[0]), w1 = __bfloat162float(e[1]), w2 = __bfloat162float(e[2]),
-                  w3 = __bfloat162float(e[3]);
-      __half* gdst = c < D ? tk + c * CH : tv + (c - D) * CH;
+      if (c < DK + dv) {
+        const int zc = c < DK ? kh * DK + c : n_k + h * dv + (c - DK);
+        const uint2 wv = *(const uint2*)(p.conv_w + (long long)(n_k + zc) * SR_CONV_W);
+        const __nv_bfloat16* e = (const __nv_bfloat16*)&wv;
+        const float w0 = __bfloat162float(e[0]), w1 = __bfloat162float(e[1]), w2 = __bfloat162float(e[2]),
+                    w3 = __bfloat162float(e[3]);
+        __half* gdst = c < DK ? tk + c * CH : tv + (c - DK) * CH;
 #pragma unroll
-      for (int rho = 0; rho < 3; ++rho) {
-        float y = w0 * zr[q][rho] + w1 * zr[q][rho + 1] + w2 * zr[q][rho + 2] + w3 * zr[q][rho + 3];
-        if (!p.act_identity) y = __fdividef(y, 1.f + __expf(-y));
-        const __half hy = __float2half_rn(y);
-        gdst[rho] = hy;
-        if (c < D) sm.Ks[c * LDK + rho] = hy;
+        for (int rho = 0; rho < 3; ++rho) {
+          float y = w0 * zr[q][rho] + w1 * zr[q][rho + 1] + w2 * zr[q][rho + 2] + w3 * zr[q][rho + 3];
+          if (!p.act_identity) y = __fdividef(y, 1.f + __expf(-y));
+          const __half hy = __float2half_rn(y);
+          gdst[rho] = hy;
+          if (c < DK) sm.Ks[c * LDK + rho] = hy;
+        }
       }
     }
     __syncthreads();
@@ -200,7 +206,7 @@ __global__ void __launch_bounds__(LT, LOCAL_CTAS_PER_SM) sr_chunk_local_kernel(c
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[cb][j][c] = 0.f;
 #pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks) {
+    for (int ks = 0; ks < DK / 16; ++ks) {
       uint32_t a[4], b[4];
       ldsm4t(a, at_addr(sm.Ks, LDK, ks * 16, rb * 16, l));
 #pragma unroll
@@ -398,207 +404,30 @@ __global__ void __launch_bounds__(LT, LOCAL_CTAS_PER_SM) sr_chunk_local_kernel(c
   }
 }
 
-// ---------------------------------------------------------------------------------------------------
-// the chain
-
-struct ChainSmem {
-  __half Ks[D * LDK];             // keys, channel-major
-  __half VU[D * LDK];             // values, channel-major; later U' as [64 rows][LDH]
-  __half Wn[CH * LDH];            // -W
-  __half S16[D * LDH];            // state as fp16 operand of W S0
-  __half Tb[CH * LDT];
-  __half Tw[CH * LDT];
-  float sc[SC_FLOATS];            // row factors exp(g_n - g_j) n_j, then gamma_n
-};
-static_assert(D * LDK >= CH * LDH, "U' must fit in the value tile's buffer");
-
-struct ChainParams {
-  SrSched s;
-  const __half* kv16;
-  const __half* tt;
-  const float* sc;
-  int32_t ncb;
-  int32_t n_k_heads, n_v_heads;
-  char* out_layer;
-  int64_t slot_stride;
-};
-
-__global__ void __launch_bounds__(THREADS, 2) sr_scan_chain_kernel(const ChainParams p) {
-  extern __shared__ __align__(16) uint8_t smem_raw[];
-  ChainSmem& sm = *reinterpret_cast<ChainSmem*>(smem_raw);
-  const int h = blockIdx.x, req = p.s.req_order[blockIdx.y];       // longest chains first
-  const int out_slot = p.s.req_out[req];
-  if (out_slot < 0) return;
-  const int R = p.s.req_rows[req];
-  const int tid = threadIdx.x, warp = tid >> 5, l = tid & 31, g8 = l >> 2, t4 = l & 3;
-  float* out = (float*)(p.out_layer + (int64_t)out_slot * p.slot_stride) + (int64_t)h * D * D;
-  const int kh = h / (p.n_v_heads / p.n_k_heads);
-  const int slot0 = p.s.req_slot0[req];
-
-  // state tile of this warp: rows mb*32 .. +31 (2 m-tiles), cols nb*64 .. +63 (8 n-tiles)
-  const int mb = warp >> 1, nb = warp & 1;
-  float accS[2][8][4];
-#pragma unroll
-  for (int a = 0; a < 2; ++a)
-#pragma unroll
-    for (int b = 0; b < 8; ++b)
-#pragma unroll
-      for (int c = 0; c < 4; ++c) accS[a][b][c] = 0.f;
-  const int rb = warp >> 1, ch = warp & 1;               // row block / column half in the 64-row products
-
-  const int n_chunks = (R + CH - 1) / CH;
-  for (int ck = 0; ck < n_chunks; ++ck) {
-    const int slot = slot0 + ck;
-    const __half* tk = p.kv16 + ((long long)slot * p.ncb + kh) * (CH * D);
-    const __half* tv = p.kv16 + ((long long)slot * p.ncb + p.n_k_heads + h) * (CH * D);
-    const __half* tt = p.tt + ((long long)slot * p.n_v_heads + h) * TT_HALFS;
-    // ---- fetch the chunk: k and v tiles, the two T matrices, the row factors ----------------------
-    for (int i = tid; i < 2 * D * (CH / 8); i += THREADS) {
-      const int which = i >> 10, c = (i >> 3) & (D - 1), seg = i & 7;
-      cp_async16((which ? sm.VU : sm.Ks) + c * LDK + seg * 8, (which ? tv : tk) + c * CH + seg * 8);
-    }
-    for (int i = tid; i < 2 * CH * (CH / 8); i += THREADS) {
-      const int which = i >> 9, r = (i >> 3) & (CH - 1), seg = i & 7;
-      cp_async16((which ? sm.Tw : sm.Tb) + r * LDT + seg * 8, tt + which * (CH * CH) + r * CH + seg * 8);
-    }
-    if (tid < (CH + 4) / 4)
-      cp_async16(sm.sc + 4 * tid, p.sc + ((long long)slot * p.n_v_heads + h) * SC_FLOATS + 4 * tid);
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    if (ck + 1 < n_chunks) {        // pull the next chunk's tiles towards L2
-      const __half* nk = tk + (long long)p.ncb * (CH * D);
-      const __half* nv = tv + (long long)p.ncb * (CH * D);
-      const __half* nt = tt + (long long)p.n_v_heads * TT_HALFS;
-      prefetch_l2((tid < 128 ? nk : nv) + (tid & 127) * 64);
-      if (tid < 128) prefetch_l2(nt + tid * 64);
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncthreads();
-
-    // ---- W = Tw K, then U~ = Tb V: warp (rb, ch) owns rows rb*16.., cols ch*64..+63 ---------------
-    float accU[8][4];
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-#pragma unroll
-      for (int c = 0; c < 4; ++c) accU[j][c] = 0.f;
-    if (ck > 0) {       // W is only needed when there is a state to read
-      for (int kb = 0; kb <= rb; ++kb) {
-        uint32_t a_w[4], b[4];
-        ldsm4t(a_w, at_addr(sm.Tw, LDT, kb * 16, rb * 16, l));
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          ldsm4(b, bn_addr(sm.Ks, LDK, ch * 64 + jj * 16, kb * 16, l));
-          mma16816(accU[2 * jj], a_w, b[0], b[1]);
-          mma16816(accU[2 * jj + 1], a_w, b[2], b[3]);
-        }
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        __half* dst = sm.Wn + (rb * 16 + g8) * LDH + ch * 64 + j * 8 + 2 * t4;
-        *(uint32_t*)dst = pack_h2(-accU[j][0], -accU[j][1]);
-        *(uint32_t*)(dst + 8 * LDH) = pack_h2(-accU[j][2], -accU[j][3]);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) accU[j][c] = 0.f;
-      }
-    }
-    for (int kb = 0; kb <= rb; ++kb) {
-      uint32_t a_b[4], b[4];
-      ldsm4t(a_b, at_addr(sm.Tb, LDT, kb * 16, rb * 16, l));
-#pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        ldsm4(b, bn_addr(sm.VU, LDK, ch * 64 + jj * 16, kb * 16, l));
-        mma16816(accU[2 * jj], a_b, b[0], b[1]);
-        mma16816(accU[2 * jj + 1], a_b, b[2], b[3]);
-      }
-    }
-    __syncthreads();     // V is dead from here on: its buffer becomes U'
-
-    // ---- U = U~ - W S0 (S0 = 0 in the first chunk), U' = row-scaled U -----------------------------
-    if (ck > 0) {
-#pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks) {
-        uint32_t a[4], b[4];
-        ldsm4(a, a_addr(sm.Wn, LDH, rb * 16, ks * 16, l));
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          ldsm4t(b, bt_addr(sm.S16, LDH, ks * 16, ch * 64 + jj * 16, l));
-          mma16816(accU[2 * jj], a, b[0], b[1]);
-          mma16816(accU[2 * jj + 1], a, b[2], b[3]);
-        }
-      }
-    }
-    {
-      const int r0 = rb * 16 + g8, r1 = r0 + 8;
-      const float s0 = sm.sc[r0], s1 = sm.sc[r1];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        __half* dst = sm.VU + r0 * LDH + ch * 64 + j * 8 + 2 * t4;
-        *(uint32_t*)dst = pack_h2(accU[j][0] * s0, accU[j][1] * s0);
-        *(uint32_t*)(dst + 8 * LDH) = pack_h2(accU[j][2] * s1, accU[j][3] * s1);
-      }
-    }
-    const float decay = sm.sc[CH];
-    __syncthreads();
-
-    // ---- S = gamma_n S + K^T U' ------------------------------------------------------------------
-#pragma unroll
-    for (int a = 0; a < 2; ++a)
-#pragma unroll
-      for (int b = 0; b < 8; ++b)
-#pragma unroll
-        for (int c = 0; c < 4; ++c) accS[a][b][c] *= decay;
-#pragma unroll
-    for (int ks = 0; ks < CH / 16; ++ks) {
-      uint32_t a0[4], a1[4], b[4];
-      ldsm4(a0, a_addr(sm.Ks, LDK, mb * 32, ks * 16, l));
-      ldsm4(a1, a_addr(sm.Ks, LDK, mb * 32 + 16, ks * 16, l));
-#pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        ldsm4t(b, bt_addr(sm.VU, LDH, ks * 16, nb * 64 + jj * 16, l));
-        mma16816(accS[0][2 * jj], a0, b[0], b[1]);
-        mma16816(accS[0][2 * jj + 1], a0, b[2], b[3]);
-        mma16816(accS[1][2 * jj], a1, b[0], b[1]);
-        mma16816(accS[1][2 * jj + 1], a1, b[2], b[3]);
-      }
-    }
-    if (ck + 1 < n_chunks) {
-#pragma unroll
-      for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          __half* dst = sm.S16 + (mb * 32 + a * 16 + g8) * LDH + nb * 64 + j * 8 + 2 * t4;
-          *(uint32_t*)dst = pack_h2(accS[a][j][0], accS[a][j][1]);
-          *(uint32_t*)(dst + 8 * LDH) = pack_h2(accS[a][j][2], accS[a][j][3]);
-        }
-    }
-    __syncthreads();   // K, U', T, S16 are rewritten by the next chunk
-  }
-
-#pragma unroll
-  for (int a = 0; a < 2; ++a)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      float* dst = out + (int64_t)(mb * 32 + a * 16 + g8) * D + nb * 64 + j * 8 + 2 * t4;
-      *(float2*)dst = make_float2(accS[a][j][0], accS[a][j][1]);
-      *(float2*)(dst + 8 * D) = make_float2(accS[a][j][2], accS[a][j][3]);
-    }
-}
-
 }  // namespace
 
 size_t sr_scan_split_bytes(const sr_ctx* ctx, int64_t max_slots) {
   return (size_t)max_slots * ctx->desc.n_v_heads * (TT_HALFS * sizeof(__half) + SC_FLOATS * sizeof(float));
 }
 
+bool sr_chunk_local_supported(int d_k, int d_v) {
+  return (d_k == 64 || d_k == 96 || d_k == 128) && d_v % 8 == 0 && d_v > 0 && d_k + d_v <= 3 * LT;
+}
+
+template <int DK>
+static cudaError_t launch_chunk_local(const LocalParams& p, dim3 grid, cudaStream_t stream) {
+  cudaError_t e = sr_once_per_device(DK == 64 ? SR_ONCE_CHUNK_LOCAL_64 : DK == 96 ? SR_ONCE_CHUNK_LOCAL_96 : SR_ONCE_CHUNK_LOCAL_128, [] {
+    return cudaFuncSetAttribute(sr_chunk_local_kernel<DK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)sizeof(LocalSmem<DK>));
+  });
+  if (e != cudaSuccess) return e;
+  sr_chunk_local_kernel<DK><<<grid, LT, sizeof(LocalSmem<DK>), stream>>>(p);
+  return cudaGetLastError();
+}
+
 cudaError_t sr_launch_chunk_local(const sr_ctx* ctx, const SrSched& s, const sr_layer_weights& w, const SrFused& fused,
                                   void* split_buf, cudaStream_t stream) {
   const sr_model_desc& d = ctx->desc;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(sr_chunk_local_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)sizeof(LocalSmem));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
   LocalParams p;
   p.s = s;
   p.gates = fused.gates;
@@ -609,6 +438,7 @@ cudaError_t sr_launch_chunk_local(const sr_ctx* ctx, const SrSched& s, const sr_
   p.fix_mod = fused.fix_mod;
   p.n_k_heads = d.n_k_heads;
   p.n_v_heads = d.n_v_heads;
+  p.d_v = d.d_v;
   p.act_identity = d.conv_activation == SR_CONV_IDENTITY;
   p.erase = d.recurrence == SR_REC_GATED_DELTA;
   p.eps = d.l2_eps;
@@ -618,31 +448,10 @@ cudaError_t sr_launch_chunk_local(const sr_ctx* ctx, const SrSched& s, const sr_
   p.tt = (__half*)split_buf;
   p.sc = (float*)((char*)split_buf + (size_t)s.max_slots * d.n_v_heads * TT_HALFS * sizeof(__half));
   dim3 grid((unsigned)d.n_v_heads, (unsigned)s.max_slots);
-  sr_chunk_local_kernel<<<grid, LT, sizeof(LocalSmem), stream>>>(p);
-  return cudaGetLastError();
-}
-
-cudaError_t sr_launch_scan_chain(const sr_ctx* ctx, const SrSched& s, const SrFused& fused, const void* split_buf,
-                                 char* out_ssm_layer, int64_t slot_stride, cudaStream_t stream) {
-  const sr_model_desc& d = ctx->desc;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(sr_scan_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)sizeof(ChainSmem));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
+  switch (d.d_k) {
+    case 64: return launch_chunk_local<64>(p, grid, stream);
+    case 96: return launch_chunk_local<96>(p, grid, stream);
+    case 128: return launch_chunk_local<128>(p, grid, stream);
+    default: return cudaErrorInvalidValue;
   }
-  ChainParams p;
-  p.s = s;
-  p.kv16 = fused.kv16;
-  p.tt = (const __half*)split_buf;
-  p.sc = (const float*)((const char*)split_buf + (size_t)s.max_slots * d.n_v_heads * TT_HALFS * sizeof(__half));
-  p.ncb = fused.ncb;
-  p.n_k_heads = d.n_k_heads;
-  p.n_v_heads = d.n_v_heads;
-  p.out_layer = out_ssm_layer;
-  p.slot_stride = slot_stride;
-  dim3 grid((unsigned)d.n_v_heads, (unsigned)s.n_requests);
-  sr_scan_chain_kernel<<<grid, THREADS, sizeof(ChainSmem), stream>>>(p);
-  return cudaGetLastError();
 }

@@ -1,4 +1,4 @@
-// Batch packing on the device (Section 5.3, "Batched replay": the replay suffixes of a batch
+// Batch packing on the device (Section 5.2, "Batched replay": the replay suffixes of a batch
 // are packed into one variable-length execution and device-side boundaries identify each
 // request's segment and destination state slot; padding segments carry a sentinel slot).
 //
@@ -15,7 +15,7 @@ constexpr int kSchedThreads = 1024;
 __global__ void __launch_bounds__(kSchedThreads)
 sr_schedule_kernel(SrSched s, const int32_t* __restrict__ pages, const int32_t* __restrict__ state_slots,
                    const int32_t* __restrict__ replay_lens, int32_t max_pages, int32_t max_replay_len,
-                   int64_t max_total_rows, int32_t n_phys_pages) {
+                   int64_t max_total_rows, int32_t n_phys_pages, int32_t n_state_slots) {
   __shared__ long long part_pages[kSchedThreads];
   __shared__ long long part_rows[kSchedThreads];
   __shared__ unsigned int flags;
@@ -31,7 +31,7 @@ sr_schedule_kernel(SrSched s, const int32_t* __restrict__ pages, const int32_t* 
     unsigned int bad = 0u;
     if (out == -1) {            // sentinel: a padding segment, silently skipped
       R = 0;
-    } else if (out < -1) {
+    } else if (out < -1 || (n_state_slots > 0 && out >= n_state_slots)) {
       bad = SR_DEV_BAD_SLOT;
     } else if (R < 0 || R > max_replay_len) {
       bad = SR_DEV_BAD_REPLAY_LEN;
@@ -164,9 +164,10 @@ sr_debug_gather_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d
 
 cudaError_t sr_launch_schedule(const SrSched& s, const int32_t* pages, const int32_t* state_slots,
                                const int32_t* replay_lens, int32_t max_pages, int32_t max_replay_len,
-                               int64_t max_total_rows, int32_t n_phys_pages, cudaStream_t stream) {
+                               int64_t max_total_rows, int32_t n_phys_pages, int32_t n_state_slots,
+                               cudaStream_t stream) {
   sr_schedule_kernel<<<1, kSchedThreads, 0, stream>>>(s, pages, state_slots, replay_lens, max_pages,
-                                                      max_replay_len, max_total_rows, n_phys_pages);
+                                                      max_replay_len, max_total_rows, n_phys_pages, n_state_slots);
   return cudaGetLastError();
 }
 

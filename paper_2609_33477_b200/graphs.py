@@ -1,4 +1,4 @@
-"""Replay graphs with static buffers (Section 5.3, "Batched replay").
+"""Replay graphs with static buffers (Section 5.2, "Batched replay"; Section 6, "Replay graphs").
 
 The replay call reads lengths, page tables and destination slots on the device and allocates nothing, so one
 captured CUDA graph serves every batch that fits the bounds it was captured with.  Grids and scratch are sized by
@@ -60,10 +60,14 @@ class BucketedGraphReplayer:
         raise ValueError(f"no bucket holds {n_requests} requests / {total_rows} rows")
 
     def replay(self, pages: torch.Tensor, lens: torch.Tensor, slots: torch.Tensor) -> int:
-        """Rebuilds the states of one batch: ``pages`` [n, <= max_pages] int32, ``lens`` [n] int32, ``slots`` [n]
-        int32 (host or device tensors).  Returns the bucket used.  Asynchronous on the current stream."""
+        """Rebuilds the states of one batch: ``pages`` [n, <= max_pages] int32 and ``slots`` [n] int32 (host or
+        device tensors), ``lens`` [n] int32 on the HOST -- the bucket is chosen from the lengths the scheduler
+        already holds, so nothing here waits for the device (the hit path adds no host synchronisation,
+        Section 5.2).  Returns the bucket used.  Asynchronous on the current stream."""
+        if lens.device.type != "cpu":
+            raise ValueError("replay lengths must be a host tensor: the bucket is picked on the host, without a device sync")
         n = int(lens.shape[0])
-        i = self.pick(n, int(lens.clamp(min=0).sum().item()))
+        i = self.pick(n, int(lens.clamp(min=0).sum()))
         b = self.buckets[i][0]
         self.slots[:b].fill_(-1)                              # padding segments: sentinel
         self.lens[:b].zero_()

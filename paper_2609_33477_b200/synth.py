@@ -88,7 +88,15 @@ SPECS = {
                                    d_k=128, d_v=128, n_requests=3, replay=("list", (130, 64, 200))),
     "wide_v_small": WorkloadSpec(name="wide_v_small", n_layers=2, d_model=256, n_k_heads=2, n_v_heads=2,
                                  d_k=96, d_v=192, n_requests=4, replay=("list", (70, 0, 129, 5)), layer_mask="even"),
-    # the per-head-decay family (no erase) on the tensor-core kernels and on the token scan
+    # head geometry of the paper's three models (Appendix A table: 16/32 heads of 128; 16/48 heads of 128; 16/16
+    # heads of 96/192), few layers, narrow d_model: parity cases
+    "geom_16_32": WorkloadSpec(name="geom_16_32", n_layers=1, d_model=256, n_k_heads=16, n_v_heads=32, d_k=128, d_v=128,
+                               n_requests=2, replay=("list", (130, 64))),
+    "geom_16_48": WorkloadSpec(name="geom_16_48", n_layers=1, d_model=256, n_k_heads=16, n_v_heads=48, d_k=128, d_v=128,
+                               n_requests=2, replay=("list", (70, 129))),
+    "geom_96_192": WorkloadSpec(name="geom_96_192", n_layers=1, d_model=256, n_k_heads=3, n_v_heads=3, d_k=96, d_v=192,
+                                n_requests=3, replay=("list", (200, 64, 321))),
+    # the per-head-decay family (no erase)
     "decay_only_small": _spec("decay_only_small", 2, 512, 4, 128, 4, ("list", (130, 64, 257, 5)), recurrence="decay_only"),
     "decay_only_d64": _spec("decay_only_d64", 1, 256, 2, 64, 3, ("list", (70, 128, 3)), recurrence="decay_only"),
     # more requests than the packing kernel has threads, many of them empty

@@ -97,6 +97,22 @@ def test_workspace_query_and_argument_checks_happen_before_any_launch(lib):
     assert st == B.SR_ERR_INVALID_ARG
     assert lib.sr_device_status(ctx, None, None, None) == B.SR_ERR_INVALID_ARG
     assert B.sr_last_launch_count(ctx) == 0
+    # a null context is an invalid argument for every entry, also where states to continue from are given
+    st = lib.sr_replay_states_from(None, C.byref(pool), C.byref(table), None, mask, weights, C.byref(out), C.byref(out),
+                                   C.byref(out), C.byref(out), None, 0, None)
+    assert st == B.SR_ERR_INVALID_ARG
+    st = lib.sr_replay_states(None, C.byref(pool), C.byref(table), None, mask, weights, C.byref(out), C.byref(out),
+                              None, 0, None)
+    assert st == B.SR_ERR_INVALID_ARG
+    B.sr_destroy(ctx)
+
+
+def test_more_requests_than_grid_rows_are_refused(lib):
+    ctx = B.sr_create(_desc())
+    n = C.c_size_t()
+    assert lib.sr_workspace_bytes(ctx, C.byref(B.sr_page_table(None, None, 65535, 0, 0, 0)), C.byref(n)) == B.SR_OK
+    assert lib.sr_workspace_bytes(ctx, C.byref(B.sr_page_table(None, None, 65536, 0, 0, 0)), C.byref(n)) == \
+        B.SR_ERR_UNSUPPORTED_SHAPE
     B.sr_destroy(ctx)
 
 

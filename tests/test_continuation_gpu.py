@@ -29,7 +29,8 @@ def _random_states(rep, seed):
     return in_ssm, in_conv
 
 
-@pytest.mark.parametrize("name", ["ragged_small", "fp8_small", "grouped_small", "decay_only_small"])
+@pytest.mark.parametrize("name", ["ragged_small", "fp8_small", "grouped_small", "decay_only_small",
+                                  "ragged_d64", "wide_v_small", "grouped3_small"])
 def test_continuation_matches_oracle(name):
     wl = synth.build_workload(name, device="cuda")
     rep = binding.Replayer(wl)
@@ -95,11 +96,3 @@ def test_zero_length_continuation_hands_the_states_through():
     for l in range(wl.spec.n_layers):
         if wl.layer_mask[l]:
             assert torch.equal(rep.out_ssm[:, l], in_ssm[:, l]) and torch.equal(rep.out_conv[:, l], in_conv[:, l])
-
-
-def test_continuation_is_refused_on_the_alternative_kernels(monkeypatch):
-    monkeypatch.setenv("SR_UNFUSED", "1")
-    wl = synth.build_workload("ragged_small", device="cuda")
-    rep = binding.Replayer(wl)
-    in_ssm, in_conv = _random_states(rep, 10)
-    assert rep.replay_states_from(in_ssm, in_conv, check=False) == 2          # SR_ERR_UNSUPPORTED_SHAPE

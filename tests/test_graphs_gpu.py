@@ -1,4 +1,6 @@
-"""Replay graphs per bucket with static buffers and sentinel padding (Section 5.3) against the direct call."""
+"""Replay graphs per bucket with static buffers and sentinel padding (Section 5.2, Section 6) against the direct call
+(a comparison of the CUDA path with itself: the direct call is compared with the CPU oracle on the same workload in
+test_parity_gpu.py)."""
 
 import pytest
 import torch
@@ -26,7 +28,8 @@ def test_bucketed_graphs_match_the_direct_call_and_pad_with_sentinels():
     total = int(wl.replay_lens.sum().item())
     runner = graphs.BucketedGraphReplayer(wl, buckets=[(2, 512), (4, 1024), (B + 3, total + 64)], n_slots=B)
     # the whole batch: only the largest bucket holds it; three padding segments ride along
-    used = runner.replay(wl.page_table, wl.replay_lens, torch.arange(B, dtype=torch.int32))
+    host_lens = wl.replay_lens.cpu()
+    used = runner.replay(wl.page_table, host_lens, torch.arange(B, dtype=torch.int32))
     torch.cuda.synchronize()
     assert used == 2 and runner.device_status(used) == 0
     for l in range(wl.spec.n_layers):
@@ -36,7 +39,7 @@ def test_bucketed_graphs_match_the_direct_call_and_pad_with_sentinels():
     runner.out_ssm.zero_()
     runner.out_conv.zero_()
     pick = [5, 1]
-    lens = wl.replay_lens[pick]
+    lens = host_lens[pick]
     used = runner.replay(wl.page_table[pick], lens, torch.tensor([0, 3], dtype=torch.int32))
     torch.cuda.synchronize()
     assert used == runner.pick(2, int(lens.sum().item())) and runner.device_status(used) == 0
@@ -47,3 +50,5 @@ def test_bucketed_graphs_match_the_direct_call_and_pad_with_sentinels():
             assert not runner.out_ssm[[1, 2, 4], l].any()          # no other slot was touched
     with pytest.raises(ValueError):
         runner.pick(B + 4, 10)
+    with pytest.raises(ValueError):                                # device-side lengths would force a host sync
+        runner.replay(wl.page_table, wl.replay_lens, torch.arange(B, dtype=torch.int32))

@@ -46,3 +46,19 @@ def test_two_ranks_reduce_time_by_max_and_sum_throughput(tmp_path):
     assert [r["total_ms"] for r in res] == [15.0, 15.0]                      # max over ranks, on every rank
     assert all(abs(r["value"] - 2 * 1000 * 4 / 15e-3) < 1e-6 for r in res)   # whole-job layer-tokens/s
     assert res[0]["shards"] == [0, 2, 4, 6] and res[1]["shards"] == [1, 3, 5]  # disjoint, covering
+
+
+def test_bench_launches_its_own_ranks_when_not_under_a_launcher():
+    """`python bench.py --gpus 2` outside torchrun starts two ranks itself; with --dry --backend gloo they only
+    rendezvous, reduce a made-up time by max and print one line from rank 0 (no GPU needed)."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "4", "--dry",
+                        "--backend", "gloo"], capture_output=True, text=True, timeout=300, env=env)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [ln for ln in p.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["dry"] is True
+    assert abs(line["ms_per_step"] - 11.0) < 1e-9            # the slower rank (10 + 1 ms per step)
+    assert abs(line["value"] - 2 * 1000 * 4 / (44.0 * 1e-3)) < 1e-6

@@ -38,7 +38,7 @@ def _active(wl):
 
 @pytest.mark.parametrize("name", ["cfg0", "ragged_d64", "ragged_small", "trunks_small", "fp8_small", "cfg1_narrow",
                                   "grouped_small", "decay_none", "decay_strong", "grouped3_small", "wide_v_small",
-                                  "decay_only_small", "decay_only_d64"])
+                                  "decay_only_small", "decay_only_d64", "geom_16_32", "geom_16_48", "geom_96_192"])
 def test_small_workloads_match_oracle_everywhere(name):
     wl, rep = _run(name)
     assert rep.device_status() == 0
@@ -139,6 +139,20 @@ def test_invalid_requests_are_skipped_and_flagged():
         assert torch.all(rep.out_ssm[bad] == 9.0) and torch.all(rep.out_conv[bad] == 9.0)
     for good in (0, 1, 4):
         U.check_request_layer(rep, wl, good, 1)
+
+
+def test_destination_slot_beyond_the_output_arrays_is_a_miss():
+    wl = synth.build_workload("ragged_d64", device=DEV)
+    slots = torch.tensor([0, 1, 7, 3, 4], dtype=torch.int32, device=DEV)      # the arrays hold 5 slots: 7 is outside
+    rep = B.Replayer(wl, state_slots=slots, n_slots=5)
+    rep.out_ssm.fill_(9.0)
+    rep.out_conv.fill_(9.0)
+    rep.replay_states()
+    torch.cuda.synchronize()
+    assert rep.device_status() == B.SR_DEV_BAD_SLOT
+    assert torch.all(rep.out_ssm[2] == 9.0) and torch.all(rep.out_conv[2] == 9.0)      # nobody wrote slot 2
+    for req in (0, 1, 3, 4):
+        U.check_request_layer(rep, wl, req, 0)
 
 
 def test_rows_beyond_the_declared_bound_are_a_miss():
@@ -270,39 +284,117 @@ def test_host_buffer_entry_with_a_row_major_pool_goes_up_in_one_piece():
         assert torch.equal(out_ssm[:, l], ref_ssm[:, l]) and torch.equal(out_conv[:, l], ref_conv[:, l])
 
 
-# ----------------------------------------------------- the alternative kernels of the same path
+# ----------------------------------------------------- second forms of single steps (debug flags)
 
-@pytest.mark.parametrize("env,name", [
-    ("SR_UNFUSED", "ragged_small"),          # tokens-on-M projection with fp32 scratch + single-kernel chunk scan
-    ("SR_UNFUSED", "fp8_small"),
-    ("SR_FP8_EXACT", "fp8_small"),
-    ("SR_SIMT_CONV_TAIL", "ragged_small"),
-    ("SR_UNFUSED", "grouped_small"),
-    ("SR_SIMT_PROJECTION", "trunks_small"),  # CUDA-core projection
-    ("SR_TOKEN_SCAN", "ragged_small"),       # token-by-token fp32 scan at d = 128
-    ("SR_MMA_SYNC_CHAIN", "trunks_small"),   # state chain on mma.sync instead of tcgen05
-    ("SR_SINGLE_CTA_MMA", "cfg1_narrow"),    # one-CTA form of the fused projection
+@pytest.mark.parametrize("flag,name", [
+    (B.SR_DEBUG_FP8_EXACT, "fp8_small"),          # fp32 promotion of bare-code partial sums, no fp16 staging
+    (B.SR_DEBUG_DOT_CONV_STATE, "ragged_small"),  # conv state by per-channel dot products
+    (B.SR_DEBUG_DOT_CONV_STATE, "fp8_small"),
+    (B.SR_DEBUG_SINGLE_CTA_MMA, "cfg1_narrow"),   # one-CTA form of the fused projection
 ])
-def test_alternative_kernels_match_oracle(monkeypatch, env, name):
-    monkeypatch.setenv(env, "1")             # read when the context is created / at launch
-    wl, rep = _run(name)
+def test_second_forms_match_oracle(flag, name):
+    wl, rep = _run(name, debug_flags=flag)
     assert rep.device_status() == 0
     for i in range(wl.spec.n_requests):
         for l in _active(wl):
             U.check_request_layer(rep, wl, i, l)
 
 
-def test_both_state_chain_kernels_agree(monkeypatch):
-    wl, rep = _run("cfg1_narrow")
-    tensor_memory = rep.out_ssm.clone()
-    monkeypatch.setenv("SR_MMA_SYNC_CHAIN", "1")
-    wl2, rep2 = _run("cfg1_narrow")
-    num = torch.linalg.matrix_norm((rep2.out_ssm - tensor_memory).double())
-    den = torch.linalg.matrix_norm(tensor_memory.double())
-    assert float((num / den).max()) < 1e-5   # same operands and roundings, different summation order
+# ----------------------------------------------------- a bounded in-kernel wait that runs out
+
+def test_an_expired_wait_raises_the_status_bit_and_leaves_the_device_usable():
+    """Fault injection without a GPU fault: with SR_DEBUG_EXPIRE_WAIT the state chain never requests the first
+    key tile and its waits give up after about a millisecond.  The kernel must then return normally: status bit
+    set, state outputs untouched, tensor memory released -- shown by a following ordinary call on the same
+    device giving the same bits as before."""
+    wl, rep = _run("ragged_small")
+    ref_ssm, ref_conv = rep.out_ssm.clone(), rep.out_conv.clone()
+    wl2 = synth.build_workload("ragged_small", device=DEV)
+    bad = B.Replayer(wl2, debug_flags=B.SR_DEBUG_EXPIRE_WAIT)
+    bad.out_ssm.fill_(5.0)
+    bad.replay_states()
+    torch.cuda.synchronize()
+    assert bad.device_status() & B.SR_DEV_WAIT_EXPIRED
+    lens = wl2.replay_lens.cpu().tolist()
+    for i, R in enumerate(lens):
+        for l in _active(wl2):
+            if R > 0:
+                assert torch.all(bad.out_ssm[i, l] == 5.0)            # a chain that gave up writes nothing
+            else:
+                assert torch.all(bad.out_ssm[i, l] == 0.0)            # nothing to wait for: zero state as usual
+    assert torch.equal(bad.out_conv, ref_conv)                        # the conv state does not pass through the chain
+    bad.close()
+    for _ in range(2):
+        rep.out_ssm.zero_()
+        rep.replay_states()
+        torch.cuda.synchronize()
+        assert rep.device_status() == 0
+        assert torch.equal(rep.out_ssm, ref_ssm) and torch.equal(rep.out_conv, ref_conv)
 
 
-# ----------------------------------------------------- graph capture (Section 5.3: replay graphs, static buffers)
+# ----------------------------------------------------- windows that end inside a page
+
+def test_rows_past_the_window_in_its_last_page_are_never_used():
+    """A window may end anywhere inside its last page (R = 65 and 200 here).  The rows behind it on that page
+    are not part of the replay -- in a live pool they are stale or not yet written -- so filling them with NaN,
+    infinities and huge values must not change one bit of the result."""
+    wl, rep = _run("ragged_small")
+    ref_ssm, ref_conv = rep.out_ssm.clone(), rep.out_conv.clone()
+    wl2 = synth.build_workload("ragged_small", device=DEV)
+    junk = torch.tensor([float("nan"), float("inf"), -float("inf"), 3.0e38], dtype=torch.bfloat16, device=DEV)
+    for i, R in enumerate(wl2.replay_lens.cpu().tolist()):
+        if R % 64:
+            page = int(wl2.page_table[i, R // 64])
+            tail = wl2.anchor_pool[page, :, R % 64:, :]
+            tail.copy_(junk[torch.arange(tail.numel(), device=DEV) % 4].view(tail.shape))
+    rep2 = B.Replayer(wl2)
+    rep2.replay_states()
+    torch.cuda.synchronize()
+    assert rep2.device_status() == 0
+    assert torch.equal(rep2.out_ssm, ref_ssm) and torch.equal(rep2.out_conv, ref_conv)
+
+
+def test_long_window_with_a_partial_last_chunk():
+    """Many full chunks followed by a partial one at d_k = d_v = 128: R = 4096 + 17 rows in one request."""
+    spec = synth.WorkloadSpec(name="long_ragged", n_layers=1, d_model=1024, n_k_heads=4, n_v_heads=4, d_k=128,
+                              d_v=128, n_requests=2, replay=("list", (4096 + 17, 64 * 3 + 63)))
+    wl = synth.build_workload(spec, device=DEV)
+    rep = B.Replayer(wl)
+    rep.replay_states()
+    torch.cuda.synchronize()
+    assert rep.device_status() == 0
+    for i in range(2):
+        U.check_request_layer(rep, wl, i, 0)
+
+
+def test_guard_bands_around_outputs_and_workspace_stay_intact():
+    """Outputs and workspace sit inside larger allocations whose margins are filled with a pattern: the call must
+    not write one byte outside the extents the boundary states (a stand-in for a memory checker)."""
+    wl = synth.build_workload("ragged_small", device=DEV)
+    s = wl.spec
+    band = 1 << 16
+    L, B_ = s.n_layers, s.n_requests
+    ssm_elems = B_ * L * s.n_v_heads * s.d_k * s.d_v
+    conv_elems = B_ * L * s.conv_channels * (s.conv_width - 1)
+    big_ssm = torch.full((ssm_elems + 2 * band,), 123.0, dtype=torch.float32, device=DEV)
+    big_conv = torch.full((conv_elems + 2 * band,), 123.0, dtype=torch.bfloat16, device=DEV)
+    out_ssm = big_ssm[band:band + ssm_elems].view(B_, L, s.n_v_heads, s.d_k, s.d_v)
+    out_conv = big_conv[band:band + conv_elems].view(B_, L, s.conv_channels, s.conv_width - 1)
+    rep = B.Replayer(wl, out_ssm=out_ssm, out_conv=out_conv)
+    big_ws = torch.full((rep.workspace_bytes + 2 * band + 256,), 0x5A, dtype=torch.uint8, device=DEV)
+    ws_ptr = (big_ws.data_ptr() + band + 255) // 256 * 256
+    off = ws_ptr - big_ws.data_ptr()
+    rep.workspace, rep._ws_ptr = big_ws, ws_ptr
+    rep.replay_states()
+    torch.cuda.synchronize()
+    assert rep.device_status() == 0
+    assert bool((big_ssm[:band] == 123.0).all()) and bool((big_ssm[band + ssm_elems:] == 123.0).all())
+    assert bool((big_conv[:band] == 123.0).all()) and bool((big_conv[band + conv_elems:] == 123.0).all())
+    assert bool((big_ws[:off] == 0x5A).all()) and bool((big_ws[off + rep.workspace_bytes:] == 0x5A).all())
+    U.check_request_layer(rep, wl, 5, 2)
+
+
+# ----------------------------------------------------- graph capture (Section 6, "Replay graphs": static buffers)
 
 def test_call_is_graph_capturable_with_device_side_boundaries():
     """The call allocates nothing, never synchronises and reads lengths, pages and slots on the device, so one
