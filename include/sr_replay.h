@@ -182,9 +182,16 @@ int sr_ssm_bytes_per_layer(const sr_ctx* ctx, size_t* out_bytes);
 /* Bytes of one layer's conv state, C*(w-1)*2 (Appendix A, B_conv). */
 int sr_conv_bytes_per_layer(const sr_ctx* ctx, size_t* out_bytes);
 
-/* Scratch bytes sr_replay_states needs for any batch within the bounds in `table`
- * (n_requests, max_pages, max_total_rows; the pointers in `table` are not read). */
+/* Scratch bytes sr_replay_states should be given for any batch within the bounds in `table`
+ * (n_requests, max_pages, max_total_rows; the pointers in `table` are not read).  The layers of one call are
+ * independent of one another (every layer has its own anchors, Eq. 2), so for a batch too small to fill the GPU
+ * with one layer the call runs up to four layers side by side, each with its own block of scratch: this size
+ * includes those blocks (as many as stay within 512 MiB together; one block for large batches). */
 int sr_workspace_bytes(const sr_ctx* ctx, const sr_page_table* table, size_t* out_bytes);
+
+/* The least scratch a call accepts for the same bounds: one block, layers one after the other.  A workspace
+ * between the two sizes is used for as many blocks as fit. */
+int sr_workspace_bytes_min(const sr_ctx* ctx, const sr_page_table* table, size_t* out_bytes);
 
 /*
  * Rebuilds the recurrent and conv state of every layer l with layer_mask[l] != 0 for every
@@ -196,8 +203,13 @@ int sr_workspace_bytes(const sr_ctx* ctx, const sr_page_table* table, size_t* ou
  *   weights      HOST   [n_layers]
  *   out_ssm      FP32, per (slot, layer): [H_v][d_k][d_v]
  *   out_conv     BF16, per (slot, layer): [C][w-1]
- *   workspace    DEVICE, 256-byte aligned, >= sr_workspace_bytes; contents are scratch.
- *                Its first word is the device status word, cleared by this call.
+ *   workspace    DEVICE, 256-byte aligned, >= sr_workspace_bytes_min (sr_workspace_bytes for full speed on
+ *                small batches); contents are scratch.  Its first word is the device status word, cleared
+ *                by this call.
+ *
+ * The call is one unit of work on `stream`: where it runs layers side by side it does so on streams of the
+ * context that fork from `stream` after the batch is packed and join it before the call's work ends (the first
+ * such call creates those streams: make it outside any stream capture).
  *
  * Outputs of masked-out layers, of sentinel requests and of skipped (invalid) requests are
  * not touched.  Results are bit-reproducible from run to run.

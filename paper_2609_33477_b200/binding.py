@@ -30,7 +30,7 @@ EXPORTS = (
     "sr_version", "sr_status_string", "sr_create", "sr_destroy", "sr_ssm_bytes_per_layer",
     "sr_conv_bytes_per_layer", "sr_workspace_bytes", "sr_replay_states", "sr_replay_states_host",
     "sr_debug_gather", "sr_device_status", "sr_last_launch_count", "sr_profile_enable", "sr_profile_read",
-    "sr_replay_states_noalloc", "sr_replay_states_from", "sr_anchor_write",
+    "sr_replay_states_noalloc", "sr_replay_states_from", "sr_anchor_write", "sr_workspace_bytes_min",
 )
 SR_NOALLOC_SCRATCH_BYTES = 128 * 1024 * 1024
 SR_KERNEL_SCHEDULE, SR_KERNEL_PROJECTION, SR_KERNEL_CONV_TAIL, SR_KERNEL_SCAN = 0, 1, 2, 3
@@ -89,6 +89,7 @@ def load() -> C.CDLL:
     lib.sr_ssm_bytes_per_layer.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
     lib.sr_conv_bytes_per_layer.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
     lib.sr_workspace_bytes.argtypes = [C.c_void_p, C.POINTER(sr_page_table), C.POINTER(C.c_size_t)]
+    lib.sr_workspace_bytes_min.argtypes = [C.c_void_p, C.POINTER(sr_page_table), C.POINTER(C.c_size_t)]
     lib.sr_replay_states.argtypes = [
         C.c_void_p, C.POINTER(sr_anchor_pool), C.POINTER(sr_page_table), C.c_void_p, C.c_void_p,
         C.POINTER(sr_layer_weights), C.POINTER(sr_out), C.POINTER(sr_out), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -163,6 +164,12 @@ def sr_conv_bytes_per_layer(ctx) -> int:
 def sr_workspace_bytes(ctx, table: sr_page_table) -> int:
     n = C.c_size_t()
     _check(load().sr_workspace_bytes(ctx, C.byref(table), C.byref(n)), "sr_workspace_bytes")
+    return n.value
+
+
+def sr_workspace_bytes_min(ctx, table: sr_page_table) -> int:
+    n = C.c_size_t()
+    _check(load().sr_workspace_bytes_min(ctx, C.byref(table), C.byref(n)), "sr_workspace_bytes_min")
     return n.value
 
 
@@ -247,7 +254,7 @@ class Replayer:
                  state_slots: Optional[torch.Tensor] = None, n_slots: Optional[int] = None,
                  max_total_rows: Optional[int] = None, max_replay_len: Optional[int] = None,
                  out_ssm: Optional[torch.Tensor] = None, out_conv: Optional[torch.Tensor] = None,
-                 debug_flags: int = 0):
+                 debug_flags: int = 0, min_workspace: bool = False):
         self.wl = workload
         spec = workload.spec
         self.spec = spec
@@ -292,7 +299,8 @@ class Replayer:
         self.out_conv = out_conv if out_conv is not None else torch.zeros(conv_shape, dtype=torch.bfloat16, device=dev)
         self._out_ssm = sr_out(self.out_ssm.data_ptr(), L * self.ssm_layer_bytes, self.ssm_layer_bytes)
         self._out_conv = sr_out(self.out_conv.data_ptr(), L * self.conv_layer_bytes, self.conv_layer_bytes)
-        self.workspace_bytes = sr_workspace_bytes(self.ctx, self.table)
+        # min_workspace: the least scratch the call accepts (layers one after the other) instead of the recommended size
+        self.workspace_bytes = (sr_workspace_bytes_min if min_workspace else sr_workspace_bytes)(self.ctx, self.table)
         self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=dev)
         self._ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
 

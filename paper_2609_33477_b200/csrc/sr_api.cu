@@ -147,6 +147,9 @@ int sr_create(const sr_model_desc* d, sr_ctx** out_ctx) {
   c->ev_used = 0;
   c->copy_in = nullptr;
   c->copy_out = nullptr;
+  c->lanes_ready = false;
+  for (int i = 0; i < SR_MAX_LANES - 1; ++i) { c->lane_stream[i] = nullptr; c->lane_join[i] = nullptr; }
+  c->lane_fork = nullptr;
   c->debug_flags = d->debug_flags;
   c->wdec_bytes = 0;
   c->kernels_cover = d->conv_width == SR_CONV_W && d->page_rows == SR_PAGE_ROWS && sr_proj_fused_supported(c) &&
@@ -166,6 +169,11 @@ void sr_destroy(sr_ctx* ctx) {
   if (!ctx) return;
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   for (cudaEvent_t e : ctx->ev_copy) cudaEventDestroy(e);
+  for (int i = 0; i < SR_MAX_LANES - 1; ++i) {
+    if (ctx->lane_stream[i]) cudaStreamDestroy(ctx->lane_stream[i]);
+    if (ctx->lane_join[i]) cudaEventDestroy(ctx->lane_join[i]);
+  }
+  if (ctx->lane_fork) cudaEventDestroy(ctx->lane_fork);
   if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
   if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
   delete ctx;
@@ -187,7 +195,16 @@ int sr_workspace_bytes(const sr_ctx* ctx, const sr_page_table* table, size_t* ou
   if (!out_bytes) return SR_ERR_INVALID_ARG;
   int st = check_batch(ctx, table);
   if (st != SR_OK) return st;
-  *out_bytes = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows).total;
+  const int lanes = sr_policy_lanes(ctx, table->n_requests, table->max_pages, table->max_total_rows);
+  *out_bytes = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, lanes).total;
+  return SR_OK;
+}
+
+int sr_workspace_bytes_min(const sr_ctx* ctx, const sr_page_table* table, size_t* out_bytes) {
+  if (!out_bytes) return SR_ERR_INVALID_ARG;
+  int st = check_batch(ctx, table);
+  if (st != SR_OK) return st;
+  *out_bytes = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, 1).total;
   return SR_OK;
 }
 
@@ -202,20 +219,19 @@ struct LayerHooks {
   bool (*after)(void* user, int layer, cudaStream_t stream);
 };
 
-int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* table, const int32_t* replay_lens,
-                const uint8_t* layer_mask, const sr_layer_weights* weights, const sr_out* out_ssm,
-                const sr_out* out_conv, void* workspace, size_t workspace_bytes, void* stream_,
-                const LayerHooks* hooks, const sr_out* in_ssm = nullptr, const sr_out* in_conv = nullptr) {
+// Every check that needs no device: run before anything is enqueued.
+int validate_call(const sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* table, const int32_t* replay_lens,
+                  const uint8_t* layer_mask, const sr_layer_weights* weights, const sr_out* out_ssm,
+                  const sr_out* out_conv, const void* workspace, size_t workspace_bytes, const sr_out* in_ssm,
+                  const sr_out* in_conv) {
   int st = check_batch(ctx, table);
   if (st != SR_OK) return st;
-  if (in_ssm || in_conv) {
-    if (in_ssm && (!in_ssm->base || !aligned(in_ssm->base, 16) || in_ssm->slot_stride_bytes % 16 ||
-                   in_ssm->layer_stride_bytes % 16))
-      return SR_ERR_INVALID_ARG;
-    if (in_conv && (!in_conv->base || !aligned(in_conv->base, 2) || in_conv->slot_stride_bytes % 2 ||
-                    in_conv->layer_stride_bytes % 2))
-      return SR_ERR_INVALID_ARG;
-  }
+  if (in_ssm && (!in_ssm->base || !aligned(in_ssm->base, 16) || in_ssm->slot_stride_bytes % 16 ||
+                 in_ssm->layer_stride_bytes % 16))
+    return SR_ERR_INVALID_ARG;
+  if (in_conv && (!in_conv->base || !aligned(in_conv->base, 2) || in_conv->slot_stride_bytes % 2 ||
+                  in_conv->layer_stride_bytes % 2))
+    return SR_ERR_INVALID_ARG;
   if (!replay_lens || !layer_mask || !weights || !out_ssm || !out_conv || !table->pages) return SR_ERR_INVALID_ARG;
   if (!out_ssm->base || !out_conv->base) return SR_ERR_INVALID_ARG;
   if (!aligned(out_ssm->base, 16) || out_ssm->slot_stride_bytes % 16 || out_ssm->layer_stride_bytes % 16)
@@ -233,33 +249,59 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
     if (d.weight_format == SR_W_E4M3_BLOCK128 && !w.w_qkv_scale) return SR_ERR_INVALID_ARG;
     if (!aligned(w.w_qkv, 16) || !aligned(w.w_ab, 16) || !aligned(w.conv_w, 16)) return SR_ERR_INVALID_ARG;
   }
-  const SrWorkspace lay = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows);
+  // the smallest workspace that serves the call holds one lane
+  const SrWorkspace lay = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, 1);
   if (!workspace || !aligned(workspace, 256) || workspace_bytes < lay.total) return SR_ERR_WORKSPACE;
+  return SR_OK;
+}
+
+// the context's lane streams and their fork / join events, made once
+bool ensure_lanes(sr_ctx* ctx) {
+  if (ctx->lanes_ready) return true;
+  for (int i = 0; i < SR_MAX_LANES - 1; ++i) {
+    if (cudaStreamCreateWithFlags(&ctx->lane_stream[i], cudaStreamNonBlocking) != cudaSuccess) return false;
+    if (cudaEventCreateWithFlags(&ctx->lane_join[i], cudaEventDisableTiming) != cudaSuccess) return false;
+  }
+  if (cudaEventCreateWithFlags(&ctx->lane_fork, cudaEventDisableTiming) != cudaSuccess) return false;
+  ctx->lanes_ready = true;
+  return true;
+}
+
+int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* table, const int32_t* replay_lens,
+                const uint8_t* layer_mask, const sr_layer_weights* weights, const sr_out* out_ssm,
+                const sr_out* out_conv, void* workspace, size_t workspace_bytes, void* stream_,
+                const LayerHooks* hooks, const sr_out* in_ssm = nullptr, const sr_out* in_conv = nullptr) {
+  int st = validate_call(ctx, pool, table, replay_lens, layer_mask, weights, out_ssm, out_conv, workspace,
+                         workspace_bytes, in_ssm, in_conv);
+  if (st != SR_OK) return st;
+  const sr_model_desc& d = ctx->desc;
   cudaStream_t stream = (cudaStream_t)stream_;
   ctx->last_launches = 0;
   ctx->ev_used = 0;
   ctx->ev_kind.clear();
   if (table->n_requests == 0) return SR_OK;
 
-  const SrSched sched = sr_sched_view(workspace, lay, table->n_requests);
+  // Layers are independent units (each has its own anchors, weights and outputs), so a batch too small to fill
+  // the device with one layer runs several layers side by side: layer j of the call goes to lane j % lanes, a
+  // lane being a stream with its own block of hand-over buffers.  As many lanes as the policy gives and the
+  // workspace holds; lane 0 is the caller's stream, the others fork from it after the packing kernel and join
+  // it at the end, so the call stays one unit of work on `stream` (and one graph when captured).
+  int n_active = 0;
+  for (int l = 0; l < d.n_layers; ++l) n_active += layer_mask[l] ? 1 : 0;
+  int lanes = sr_policy_lanes(ctx, table->n_requests, table->max_pages, table->max_total_rows);
+  while (lanes > 1 && (lanes > n_active ||
+                       sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, lanes).total > workspace_bytes))
+    lanes >>= 1;
+  const SrWorkspace lay = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, lanes);
+  if (lanes > 1 && !ensure_lanes(ctx)) return SR_ERR_CUDA;
+
+  SrSched sched = sr_sched_view(workspace, lay, table->n_requests);
+  sched.check_bounds = (ctx->debug_flags & SR_DEBUG_CHECK_BOUNDS) ? 1 : 0;
+  sched.n_phys_pages = pool->n_phys_pages;
+  sched.n_state_slots = table->n_state_slots;
   const SrPoolView pv = pool_view(pool);
-  float* z = (float*)((char*)workspace + lay.off_z);
   int sm_count = 0;
   if (sr_current_device_sms(&sm_count) != cudaSuccess) return SR_ERR_CUDA;
-  SrFused fused_buf;
-  fused_buf.kv16 = (__half*)((char*)workspace + lay.off_kv16);
-  fused_buf.zraw = (float*)((char*)workspace + lay.off_zraw);
-  fused_buf.gates = z;
-  fused_buf.ncb = (ctx->n_k + ctx->n_v + 127) / 128;
-  fused_buf.n_kv = ctx->n_k + ctx->n_v;
-  fused_buf.n_gate = ctx->n_gate;
-  fused_buf.fix_mod = (d.weight_format == SR_W_E4M3_BLOCK128 && !ctx->fp16_stage) ? 2 : 4;
-  fused_buf.hist = nullptr;
-  fused_buf.in_ssm_layer = nullptr;
-  fused_buf.in_ssm_slot_stride = 0;
-  fused_buf.x16 = ctx->fp16_stage ? (const __half*)((char*)workspace + lay.off_x16) : nullptr;
-  fused_buf.w16 = ctx->fp16_stage ? (const __half*)((char*)workspace + lay.off_wdec) : nullptr;
-  const SrFused& fused = fused_buf;
 
   {
     LaunchScope scope(ctx, stream, SR_KERNEL_SCHEDULE);
@@ -268,62 +310,92 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
                            stream) != cudaSuccess)
       return SR_ERR_CUDA;
   }
-  for (int l = 0; l < d.n_layers; ++l) {
+  if (lanes > 1) {
+    if (cudaEventRecord(ctx->lane_fork, stream) != cudaSuccess) return SR_ERR_CUDA;
+    for (int i = 0; i < lanes - 1; ++i)
+      if (cudaStreamWaitEvent(ctx->lane_stream[i], ctx->lane_fork, 0) != cudaSuccess) return SR_ERR_CUDA;
+  }
+  int status = SR_OK, j = 0;
+  for (int l = 0; l < d.n_layers && status == SR_OK; ++l) {
     if (!layer_mask[l]) continue;
+    const int lane = j++ % lanes;
+    cudaStream_t ls = lane == 0 ? stream : ctx->lane_stream[lane - 1];
+    char* base = (char*)workspace + (size_t)lane * lay.lane_bytes;       // this lane's hand-over block
+    SrFused fused;
+    fused.kv16 = (__half*)(base + lay.off_kv16);
+    fused.zraw = (float*)(base + lay.off_zraw);
+    fused.gates = (float*)(base + lay.off_z);
+    fused.ncb = (ctx->n_k + ctx->n_v + 127) / 128;
+    fused.n_kv = ctx->n_k + ctx->n_v;
+    fused.n_gate = ctx->n_gate;
+    fused.fix_mod = (d.weight_format == SR_W_E4M3_BLOCK128 && !ctx->fp16_stage) ? 2 : 4;
+    fused.hist = nullptr;
+    fused.in_ssm_layer = nullptr;
+    fused.in_ssm_slot_stride = 0;
+    fused.x16 = ctx->fp16_stage ? (const __half*)(base + lay.off_x16) : nullptr;
+    fused.w16 = ctx->fp16_stage ? (const __half*)(base + lay.off_wdec) : nullptr;
     const int pl = pool->layer_to_pool[l];
     char* ssm_l = (char*)out_ssm->base + (int64_t)l * out_ssm->layer_stride_bytes;
     char* conv_l = (char*)out_conv->base + (int64_t)l * out_conv->layer_stride_bytes;
-    void* wdec = (char*)workspace + lay.off_wdec;
-    if (hooks && !hooks->before(hooks->user, l, pl, stream)) return SR_ERR_CUDA;
-    if (in_conv) {
-      __nv_bfloat16* hist = (__nv_bfloat16*)((char*)workspace + lay.off_hist);
-      LaunchScope scope(ctx, stream, SR_KERNEL_CONV_TAIL);
-      if (sr_launch_hist_gather(ctx, sched, (const char*)in_conv->base + (int64_t)l * in_conv->layer_stride_bytes,
-                                in_conv->slot_stride_bytes, hist, stream) != cudaSuccess)
-        return SR_ERR_CUDA;
-      fused_buf.hist = hist;
-    }
-    if (in_ssm) {
-      fused_buf.in_ssm_layer = (const char*)in_ssm->base + (int64_t)l * in_ssm->layer_stride_bytes;
-      fused_buf.in_ssm_slot_stride = in_ssm->slot_stride_bytes;
-    }
-    if (ctx->fp16_stage) {
-      {
-        LaunchScope scope(ctx, stream, SR_KERNEL_WEIGHT_DECODE);
-        if (sr_launch_stage_weights_fp16(ctx, weights[l], (__half*)wdec, stream) != cudaSuccess) return SR_ERR_CUDA;
+    void* wdec = base + lay.off_wdec;
+    void* split = base + lay.off_split;
+    status = SR_ERR_CUDA;       // any early exit below is a failed CUDA call; the lanes are still joined
+    do {
+      if (hooks && !hooks->before(hooks->user, l, pl, ls)) break;
+      if (in_conv) {
+        __nv_bfloat16* hist = (__nv_bfloat16*)(base + lay.off_hist);
+        LaunchScope scope(ctx, ls, SR_KERNEL_CONV_TAIL);
+        if (sr_launch_hist_gather(ctx, sched, (const char*)in_conv->base + (int64_t)l * in_conv->layer_stride_bytes,
+                                  in_conv->slot_stride_bytes, hist, ls) != cudaSuccess)
+          break;
+        fused.hist = hist;
       }
-      LaunchScope scope(ctx, stream, SR_KERNEL_ANCHOR_STAGE);
-      if (sr_launch_stage_anchors_fp16(ctx, sched, pv, pl, (__half*)((char*)workspace + lay.off_x16), stream) != cudaSuccess)
-        return SR_ERR_CUDA;
-    } else if (ctx->wdec_bytes) {
-      LaunchScope scope(ctx, stream, SR_KERNEL_WEIGHT_DECODE);
-      if (sr_launch_weight_decode(ctx, weights[l], wdec, stream) != cudaSuccess) return SR_ERR_CUDA;
-    }
-    {
-      LaunchScope scope(ctx, stream, SR_KERNEL_PROJECTION);
-      if (sr_launch_proj_fused(ctx, sched, *pool, pl, weights[l], ctx->wdec_bytes ? wdec : nullptr, fused, sm_count,
-                               stream) != cudaSuccess)
-        return SR_ERR_CUDA;
-    }
-    {
-      LaunchScope scope(ctx, stream, SR_KERNEL_CONV_TAIL, sr_conv_tail_launches(ctx));
-      if (sr_launch_conv_tail(ctx, sched, pv, pl, weights[l], fused, conv_l, out_conv->slot_stride_bytes, stream) !=
-          cudaSuccess)
-        return SR_ERR_CUDA;
-    }
-    {
-      void* split = (char*)workspace + lay.off_split;
-      {
-        LaunchScope scope(ctx, stream, SR_KERNEL_CHUNK_LOCAL);
-        if (sr_launch_chunk_local(ctx, sched, weights[l], fused, split, stream) != cudaSuccess) return SR_ERR_CUDA;
+      if (in_ssm) {
+        fused.in_ssm_layer = (const char*)in_ssm->base + (int64_t)l * in_ssm->layer_stride_bytes;
+        fused.in_ssm_slot_stride = in_ssm->slot_stride_bytes;
       }
-      LaunchScope scope(ctx, stream, SR_KERNEL_SCAN);
-      if (sr_launch_scan_chain_umma(ctx, sched, fused, split, ssm_l, out_ssm->slot_stride_bytes, sm_count, stream) != cudaSuccess)
-        return SR_ERR_CUDA;
-    }
-    if (hooks && !hooks->after(hooks->user, l, stream)) return SR_ERR_CUDA;
+      if (ctx->fp16_stage) {
+        {
+          LaunchScope scope(ctx, ls, SR_KERNEL_WEIGHT_DECODE);
+          if (sr_launch_stage_weights_fp16(ctx, weights[l], (__half*)wdec, ls) != cudaSuccess) break;
+        }
+        LaunchScope scope(ctx, ls, SR_KERNEL_ANCHOR_STAGE);
+        if (sr_launch_stage_anchors_fp16(ctx, sched, pv, pl, (__half*)(base + lay.off_x16), ls) != cudaSuccess) break;
+      } else if (ctx->wdec_bytes) {
+        LaunchScope scope(ctx, ls, SR_KERNEL_WEIGHT_DECODE);
+        if (sr_launch_weight_decode(ctx, weights[l], wdec, ls) != cudaSuccess) break;
+      }
+      {
+        LaunchScope scope(ctx, ls, SR_KERNEL_PROJECTION);
+        if (sr_launch_proj_fused(ctx, sched, *pool, pl, weights[l], ctx->wdec_bytes ? wdec : nullptr, fused, sm_count,
+                                 ls) != cudaSuccess)
+          break;
+      }
+      {
+        LaunchScope scope(ctx, ls, SR_KERNEL_CONV_TAIL, sr_conv_tail_launches(ctx, sched.n_requests));
+        if (sr_launch_conv_tail(ctx, sched, pv, pl, weights[l], fused, conv_l, out_conv->slot_stride_bytes, ls) !=
+            cudaSuccess)
+          break;
+      }
+      {
+        LaunchScope scope(ctx, ls, SR_KERNEL_CHUNK_LOCAL);
+        if (sr_launch_chunk_local(ctx, sched, weights[l], fused, split, ls) != cudaSuccess) break;
+      }
+      {
+        LaunchScope scope(ctx, ls, SR_KERNEL_SCAN);
+        if (sr_launch_scan_chain_umma(ctx, sched, fused, split, ssm_l, out_ssm->slot_stride_bytes, sm_count, ls) != cudaSuccess)
+          break;
+      }
+      if (hooks && !hooks->after(hooks->user, l, ls)) break;
+      status = SR_OK;
+    } while (false);
   }
-  return SR_OK;
+  // join: whatever happened above, `stream` resumes only after every lane's work
+  for (int i = 0; i < lanes - 1; ++i)
+    if (cudaEventRecord(ctx->lane_join[i], ctx->lane_stream[i]) != cudaSuccess ||
+        cudaStreamWaitEvent(stream, ctx->lane_join[i], 0) != cudaSuccess)
+      status = SR_ERR_CUDA;
+  return status;
 }
 }  // namespace
 
@@ -431,7 +503,9 @@ int sr_replay_states_host(sr_ctx* ctx, const void* host_pool, size_t pool_bytes,
       !out_ssm || !out_conv || !host_out_ssm || !host_out_conv || !layer_mask)
     return SR_ERR_INVALID_ARG;
   if ((host_state_slots == nullptr) != (table->state_slots == nullptr)) return SR_ERR_INVALID_ARG;
-  st = check_pool(ctx, pool);
+  // everything the host can check, before the first copy is enqueued
+  st = validate_call(ctx, pool, table, dev_replay_lens, layer_mask, weights, out_ssm, out_conv, workspace, workspace_bytes,
+                     nullptr, nullptr);
   if (st != SR_OK) return st;
   cudaStream_t stream = (cudaStream_t)stream_;
   if (!ctx->copy_in && cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking) != cudaSuccess) return SR_ERR_CUDA;
@@ -506,14 +580,14 @@ int sr_replay_states_host(sr_ctx* ctx, const void* host_pool, size_t pool_bytes,
   LayerHooks hooks = {&hp, pipe_before, pipe_after};
   st = replay_impl(ctx, pool, table, dev_replay_lens, layer_mask, weights, out_ssm, out_conv, workspace, workspace_bytes,
                    stream_, &hooks);
-  if (st != SR_OK) return st;
-  // layers that were not rebuilt are not copied back; `stream` resumes when both copy streams are done
+  // layers that were not rebuilt are not copied back; `stream` resumes when both copy streams are done -- also
+  // after a failed launch, so that no copy of this call is left running behind the caller's back
   cudaEvent_t in_done = pipe_event(ctx, hp.next_event++), out_done = pipe_event(ctx, hp.next_event++);
   if (!in_done || !out_done || cudaEventRecord(in_done, ctx->copy_in) != cudaSuccess ||
       cudaEventRecord(out_done, ctx->copy_out) != cudaSuccess || cudaStreamWaitEvent(stream, in_done, 0) != cudaSuccess ||
       cudaStreamWaitEvent(stream, out_done, 0) != cudaSuccess)
     return SR_ERR_CUDA;
-  return SR_OK;
+  return st;
 }
 
 int sr_anchor_write(sr_ctx* ctx, const sr_anchor_pool* pool, const int32_t* pool_layers, int32_t n_layers,
@@ -551,7 +625,9 @@ int sr_debug_gather(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table
   cudaStream_t stream = (cudaStream_t)stream_;
   ctx->last_launches = 0;
   if (table->n_requests == 0 || table->max_pages == 0) return SR_OK;
-  const SrSched sched = sr_sched_view(workspace, lay, table->n_requests);
+  SrSched sched = sr_sched_view(workspace, lay, table->n_requests);
+  sched.check_bounds = (ctx->debug_flags & SR_DEBUG_CHECK_BOUNDS) ? 1 : 0;
+  sched.n_phys_pages = pool->n_phys_pages;
   ctx->ev_used = 0;
   ctx->ev_kind.clear();
   if (sr_launch_schedule(sched, table->pages, table->state_slots, replay_lens, table->max_pages,

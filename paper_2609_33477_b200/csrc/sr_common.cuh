@@ -15,6 +15,8 @@
 
 #define SR_PAGE_ROWS 64
 #define SR_CONV_W 4
+#define SR_MAX_LANES 4                       // layers in flight at once on small batches
+#define SR_LANES_BUDGET_BYTES (512ull << 20) // ... as long as their hand-over buffers together stay below this
 
 struct sr_ctx {
   sr_model_desc desc;
@@ -32,6 +34,11 @@ struct sr_ctx {
   // optional per-kernel timing (sr_profile_*): events bracketing every launch of the last call
   bool profiling;
   std::vector<cudaEvent_t> ev_pool;   // created on demand, reused, destroyed with the context
+  // small batches: layers are independent, so up to SR_MAX_LANES of them run side by side on streams of the
+  // context (lane 0 is the caller's stream); created at the first call that uses them
+  cudaStream_t lane_stream[3];
+  cudaEvent_t lane_fork, lane_join[3];
+  bool lanes_ready;
   // sr_replay_states_host only: two copy streams and their events, created at its first call
   cudaStream_t copy_in, copy_out;
   std::vector<cudaEvent_t> ev_copy;
@@ -72,6 +79,8 @@ struct SrWorkspace {
   size_t off_wdec;       // [n_k + n_v (+ 2 H_v)][d_model] 16-bit decoded weights of the current layer (0 bytes for bf16 weights)
   size_t off_hist;       // bf16 [n_requests][C][w-1] conv state each request continues from (current layer)
   size_t off_x16;        // fp16 staging: half [max_slots][64][d_model] anchors of the current layer, slot order
+  size_t lane_bytes;     // size of one lane's block of hand-over buffers (off_kv16 .. end)
+  int lanes;             // lane blocks in `total`
   size_t total;
   int64_t max_slots;
 };
@@ -79,7 +88,7 @@ struct SrWorkspace {
 static inline size_t sr_align256(size_t x) { return (x + 255) & ~size_t(255); }
 
 static inline SrWorkspace sr_workspace_layout(const sr_ctx* ctx, int32_t n_requests, int32_t max_pages,
-                                              int64_t max_total_rows) {
+                                              int64_t max_total_rows, int lanes = 1) {
   SrWorkspace w;
   int64_t by_rows = max_total_rows / SR_PAGE_ROWS + n_requests;
   int64_t by_table = (int64_t)n_requests * max_pages;
@@ -96,6 +105,9 @@ static inline SrWorkspace sr_workspace_layout(const sr_ctx* ctx, int32_t n_reque
   w.off_slot_page = at; at = sr_align256(at + sizeof(int32_t) * (size_t)w.max_slots);
   w.off_slot_rows = at; at = sr_align256(at + sizeof(int32_t) * (size_t)w.max_slots);
   w.off_slot_first = at; at = sr_align256(at + sizeof(int32_t) * (size_t)w.max_slots);
+  // from here on: the per-layer hand-over buffers of lane 0; lane i sits lane_bytes * i further on
+  at = (at + 1023) & ~size_t(1023);
+  const size_t lane0 = at;
   const size_t n_kv = (size_t)ctx->n_k + ctx->n_v;
   const size_t kv_pitch = (n_kv + 127) / 128 * 128;     // channels per slot in the hand-over tiles (whole 128-channel tiles)
   w.off_kv16 = at;      at = sr_align256(at + sizeof(uint16_t) * (size_t)w.max_slots * SR_PAGE_ROWS * kv_pitch);
@@ -106,8 +118,21 @@ static inline SrWorkspace sr_workspace_layout(const sr_ctx* ctx, int32_t n_reque
   w.off_hist = at;      at = sr_align256(at + sizeof(uint16_t) * (size_t)n_requests * ctx->conv_ch * (SR_CONV_W - 1));
   w.off_x16 = at;       at = sr_align256(at + (ctx->fp16_stage ? sizeof(uint16_t) * (size_t)w.max_slots * SR_PAGE_ROWS *
                                                                      (size_t)ctx->desc.d_model : 0));
-  w.total = at;
+  at = (at + 1023) & ~size_t(1023);
+  w.lane_bytes = at - lane0;
+  w.lanes = lanes < 1 ? 1 : lanes;
+  w.total = lane0 + w.lane_bytes * (size_t)w.lanes;
   return w;
+}
+
+// Layers in flight at once for a batch of these bounds: as many (up to SR_MAX_LANES, and no more than the model has
+// layers) as keep the hand-over buffers together within SR_LANES_BUDGET_BYTES; large batches fill the device with
+// one layer and get one lane.
+static inline int sr_policy_lanes(const sr_ctx* ctx, int32_t n_requests, int32_t max_pages, int64_t max_total_rows) {
+  const size_t per_lane = sr_workspace_layout(ctx, n_requests, max_pages, max_total_rows, 1).lane_bytes;
+  int lanes = SR_MAX_LANES;
+  while (lanes > 1 && ((size_t)lanes * per_lane > SR_LANES_BUDGET_BYTES || lanes > ctx->desc.n_layers)) lanes >>= 1;
+  return lanes;
 }
 
 // Device views handed to the kernels.
@@ -123,7 +148,25 @@ struct SrSched {
   int32_t* slot_first;
   int32_t n_requests;
   int32_t max_slots;
+  // SR_DEBUG_CHECK_BOUNDS: kernels test every table-driven index against these before using it
+  int32_t check_bounds;   // 0 = off
+  int32_t n_phys_pages;   // pool pages
+  int32_t n_state_slots;  // slots in the output arrays (0 = not stated: not checked)
 };
+
+#ifdef __CUDACC__
+// Range check used under SR_DEBUG_CHECK_BOUNDS: records the failure and tells the caller to skip the access.
+__device__ __forceinline__ bool sr_check(const SrSched& s, bool in_range) {
+  if (!s.check_bounds || in_range) return true;
+  atomicOr(s.status, SR_DEV_BOUNDS_CHECK);
+  return false;
+}
+__device__ __forceinline__ bool sr_check_slot(const SrSched& s, int slot) { return sr_check(s, slot >= 0 && slot < s.max_slots); }
+__device__ __forceinline__ bool sr_check_page(const SrSched& s, int page) { return sr_check(s, page >= 0 && page < s.n_phys_pages); }
+__device__ __forceinline__ bool sr_check_out(const SrSched& s, int out_slot) {
+  return sr_check(s, out_slot >= 0 && (s.n_state_slots <= 0 || out_slot < s.n_state_slots));
+}
+#endif
 
 static inline SrSched sr_sched_view(void* workspace, const SrWorkspace& w, int32_t n_requests) {
   char* b = (char*)workspace;
@@ -139,6 +182,9 @@ static inline SrSched sr_sched_view(void* workspace, const SrWorkspace& w, int32
   s.slot_first = (int32_t*)(b + w.off_slot_first);
   s.n_requests = n_requests;
   s.max_slots = (int32_t)w.max_slots;
+  s.check_bounds = 0;
+  s.n_phys_pages = 0;
+  s.n_state_slots = 0;
   return s;
 }
 
@@ -209,7 +255,7 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
                                  cudaStream_t stream);
 
 // Conv state: last w-1 projection rows of every channel, rounded to bf16.
-int sr_conv_tail_launches(const sr_ctx* ctx);
+int sr_conv_tail_launches(const sr_ctx* ctx, int n_requests);
 cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoolView& pool, int32_t pool_layer,
                                 const sr_layer_weights& w, const SrFused& fused, char* out_conv_layer,
                                 int64_t slot_stride, cudaStream_t stream);

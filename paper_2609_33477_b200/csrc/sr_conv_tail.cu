@@ -33,6 +33,7 @@ sr_conv_tail_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_mo
   if (c >= conv_ch) return;
   const int R = s.req_rows[i];
   const int slot0 = s.req_slot0[i];
+  if (!sr_check_out(s, out_slot) || (R > 0 && !sr_check_slot(s, slot0 + (R - 1) / SR_PAGE_ROWS))) return;
   float val[SR_CONV_W - 1];
 #pragma unroll
   for (int j = 0; j < SR_CONV_W - 1; ++j) val[j] = 0.f;
@@ -57,8 +58,9 @@ sr_conv_tail_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_mo
       rows[j] = nullptr;
       if (t >= 0) {
         const int slot = slot0 + t / SR_PAGE_ROWS;
-        rows[j] = pool.base + (int64_t)s.slot_page[slot] * pool.page_stride + (int64_t)pool_layer * pool.layer_stride +
-                  (int64_t)(t % SR_PAGE_ROWS) * pool.row_stride;
+        if (sr_check_page(s, s.slot_page[slot]))
+          rows[j] = pool.base + (int64_t)s.slot_page[slot] * pool.page_stride + (int64_t)pool_layer * pool.layer_stride +
+                    (int64_t)(t % SR_PAGE_ROWS) * pool.row_stride;
       }
     }
     float acc[SR_CONV_W - 1];
@@ -141,8 +143,9 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
       const int t = s.req_rows[i] - (SR_CONV_W - 1) + j;
       if (t >= 0) {
         const int slot = s.req_slot0[i] + t / SR_PAGE_ROWS;
-        src = pool.base + (int64_t)s.slot_page[slot] * pool.page_stride + (int64_t)pool_layer * pool.layer_stride +
-              (int64_t)(t % SR_PAGE_ROWS) * pool.row_stride;
+        if (sr_check_slot(s, slot) && sr_check_page(s, s.slot_page[slot]))
+          src = pool.base + (int64_t)s.slot_page[slot] * pool.page_stride + (int64_t)pool_layer * pool.layer_stride +
+                (int64_t)(t % SR_PAGE_ROWS) * pool.row_stride;
       }
     }
     xrow[q] = src + seg * 16;
@@ -219,7 +222,7 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
     const int gr = r0 + warp * 16 + g8 + 8 * hr, i = gr / (SR_CONV_W - 1), j = gr % (SR_CONV_W - 1);
     if (i >= s.n_requests) continue;
     const int out_slot = s.req_out[i];
-    if (out_slot < 0) continue;
+    if (out_slot < 0 || !sr_check_out(s, out_slot)) continue;
     const int t = s.req_rows[i] - (SR_CONV_W - 1) + j;
     // rows before the window: zero, or the inputs of the state this request continues (kept bit for bit)
     const __nv_bfloat16* old = (t < 0 && hist) ? hist + (int64_t)i * conv_ch * (SR_CONV_W - 1) + (SR_CONV_W - 1 + t) : nullptr;
@@ -251,6 +254,7 @@ sr_conv_tail_kv_kernel(SrSched s, int32_t n_q, int32_t conv_ch, const float* __r
   if (ckv >= n_kv) return;
   const int c = n_q + ckv;
   const int R = s.req_rows[i], slot0 = s.req_slot0[i];
+  if (!sr_check_out(s, out_slot) || (R > 0 && !sr_check_slot(s, slot0 + (R - 1) / SR_PAGE_ROWS))) return;
   __nv_bfloat16* dst = (__nv_bfloat16*)(out_layer + (int64_t)out_slot * slot_stride) + (int64_t)c * (SR_CONV_W - 1);
 #pragma unroll
   for (int j = 0; j < SR_CONV_W - 1; ++j) {
@@ -282,14 +286,19 @@ sr_hist_gather_kernel(SrSched s, const char* __restrict__ in_layer, int64_t slot
 
 // kernels one sr_launch_conv_tail call launches: bf16 weights, the batched q GEMM plus the k | v copy; block-scaled
 // weights, one GEMM over all channels; geometries the 64-wide tiles do not divide, the single dot-product kernel
-static bool conv_tail_gemm_fits(const sr_ctx* ctx) {
+// The GEMM reads every weight once per 64 tail rows but walks d_model serially in one CTA per 64 channels; below
+// GEMM_MIN_REQUESTS requests the dot-product kernel (a warp per channel and request, thousands of short chains)
+// finishes sooner.
+constexpr int GEMM_MIN_REQUESTS = 16;
+
+static bool conv_tail_gemm_fits(const sr_ctx* ctx, int n_requests) {
   const bool fp8 = ctx->desc.weight_format == SR_W_E4M3_BLOCK128;
   return (fp8 ? ctx->conv_ch : ctx->n_k) % QT == 0 && ctx->desc.d_model % (fp8 ? 128 : QT) == 0 &&
-         !(ctx->debug_flags & SR_DEBUG_DOT_CONV_STATE);
+         n_requests >= GEMM_MIN_REQUESTS && !(ctx->debug_flags & SR_DEBUG_DOT_CONV_STATE);
 }
 
-int sr_conv_tail_launches(const sr_ctx* ctx) {
-  if (!conv_tail_gemm_fits(ctx)) return 1;
+int sr_conv_tail_launches(const sr_ctx* ctx, int n_requests) {
+  if (!conv_tail_gemm_fits(ctx, n_requests)) return 1;
   return ctx->desc.weight_format == SR_W_E4M3_BLOCK128 ? 1 : 2;
 }
 
@@ -302,7 +311,7 @@ cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoo
   const int tail_rows = s.n_requests * (SR_CONV_W - 1);
   if (ctx->desc.weight_format == SR_W_E4M3_BLOCK128) {
     // every channel from codes and scales in fp32: the conv state never sees a rounded weight
-    if (conv_tail_gemm_fits(ctx)) {
+    if (conv_tail_gemm_fits(ctx, s.n_requests)) {
       dim3 g((unsigned)(ctx->conv_ch / QT), (unsigned)((tail_rows + QT - 1) / QT));
       sr_conv_tail_gemm_kernel<true><<<g, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
                                                             w.w_qkv_scale, hist, out_conv_layer, slot_stride);
@@ -317,7 +326,7 @@ cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoo
   // bf16 weights: the q channels as one batched GEMM (or by dot products), the k and v channels copied from the
   // raw rows the projection kept
   const int n_q = ctx->n_k;
-  if (conv_tail_gemm_fits(ctx)) {
+  if (conv_tail_gemm_fits(ctx, s.n_requests)) {
     dim3 gq((unsigned)(n_q / QT), (unsigned)((tail_rows + QT - 1) / QT));
     sr_conv_tail_gemm_kernel<false><<<gq, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
                                                              nullptr, hist, out_conv_layer, slot_stride);

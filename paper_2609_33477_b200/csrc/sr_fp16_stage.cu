@@ -67,7 +67,7 @@ sr_decode_e4m3_kernel(const uint8_t* __restrict__ codes, __nv_bfloat16* __restri
 __global__ void __launch_bounds__(256)
 sr_stage_anchors_fp16_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_model, __half* __restrict__ x16) {
   const int slot = blockIdx.x;
-  if (slot >= (int)s.status[1] || s.slot_rows[slot] == 0) return;
+  if (slot >= (int)s.status[1] || s.slot_rows[slot] == 0 || !sr_check_page(s, s.slot_page[slot])) return;
   const char* page = pool.base + (int64_t)s.slot_page[slot] * pool.page_stride + (int64_t)pool_layer * pool.layer_stride;
   __half* dst = x16 + (int64_t)slot * SR_PAGE_ROWS * d_model;
   const int per_row = d_model / 8;

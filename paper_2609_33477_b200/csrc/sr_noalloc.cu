@@ -46,9 +46,12 @@ extern "C" int sr_replay_states_noalloc(sr_ctx* ctx, const sr_anchor_pool* pool,
                                         const sr_layer_weights* weights, const sr_out* out_ssm,
                                         const sr_out* out_conv, void* stream) {
   size_t need = 0;
-  int st = sr_workspace_bytes(ctx, table, &need);
+  int st = sr_workspace_bytes(ctx, table, &need);       // checks `ctx` and the bounds in `table`
   if (st != SR_OK) return st;
-  // the batch bounds in `table` need more scratch than the fixed array holds: refuse, launch nothing
+  // what the call cannot do without: the tables and ONE block of per-layer hand-over buffers (sr_workspace_bytes
+  // asks for up to four blocks on small batches, to run layers side by side; this entry uses as many as fit).
+  // If even that is more than the fixed array holds: refuse, launch nothing.
+  need = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, 1).total;
   if (need > (size_t)SR_NOALLOC_SCRATCH_BYTES) return SR_ERR_WORKSPACE;
   void* scratch = nullptr;
   st = scratch_for_current_device(&scratch);

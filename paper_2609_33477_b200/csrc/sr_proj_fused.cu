@@ -79,6 +79,7 @@ __device__ __forceinline__ void emit_slot(const FusedParams& p, bool gate, int c
       if (i >= vr) v[i] = 0.f;
   }
   if (!gate && ch >= p.n_kv) return;     // the last channel tile may reach past the k | v block
+  if (!sr_check_slot(p.s, slot)) return;
   if (gate) {
     if (ch < p.n_gate) {
       float* g = p.gates + ((long long)slot * p.n_gate + ch) * SR_PAGE_ROWS;
@@ -401,7 +402,11 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         int pt, tt;
         tile_coords(tile, pt, tt);
         const int slot_a = SLOTS * tt + 2 * rank;
-        const int page0 = p.fp16_stage ? slot_a : p.s.slot_page[slot_a], page1 = p.fp16_stage ? slot_a + 1 : p.s.slot_page[slot_a + 1];
+        int page0 = p.fp16_stage ? slot_a : p.s.slot_page[slot_a], page1 = p.fp16_stage ? slot_a + 1 : p.s.slot_page[slot_a + 1];
+        if (!p.fp16_stage && p.s.check_bounds) {      // a bad page id would only read the fill value (TMA clips), but say so
+          if (!sr_check_page(p.s, page0)) page0 = 0;
+          if (!sr_check_page(p.s, page1)) page1 = 0;
+        }
         const bool gate = pt == n_pt;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, p.s.status)) { ok = false; break; }

@@ -135,9 +135,11 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   const int h = blockIdx.x, req = p.s.req_order[blockIdx.y];       // longest chains first
+  if (!sr_check(p.s, req >= 0 && req < p.s.n_requests)) return;
   const int out_slot = p.s.req_out[req];
   if (out_slot < 0) return;
   const int R = p.s.req_rows[req];
+  if (!sr_check_out(p.s, out_slot) || (R > 0 && !sr_check_slot(p.s, p.s.req_slot0[req] + (R - 1) / CH))) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int dk = p.d_k, dv = p.d_v, dvb = p.dvb, col0 = (int)blockIdx.z * dvb;     // this CTA: value columns col0 .. col0 + dvb
   const int64_t head_off = (int64_t)h * dk * dv + col0;

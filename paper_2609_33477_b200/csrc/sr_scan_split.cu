@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(LT, LOCAL_CTAS_PER_SM) sr_chunk_local_kernel(c
   extern __shared__ __align__(16) uint8_t smem_raw[];
   LocalSmem<DK>& sm = *reinterpret_cast<LocalSmem<DK>*>(smem_raw);
   const int h = blockIdx.x, slot = blockIdx.y;
-  if (slot >= (int)p.s.status[1]) return;
+  if (slot >= (int)p.s.status[1] || !sr_check_slot(p.s, slot)) return;
   const int vr = p.s.slot_rows[slot];
   if (vr == 0) return;                                   // padding slot
   const int tid = threadIdx.x, warp = tid >> 5, l = tid & 31, g8 = l >> 2, t4 = l & 3;

@@ -147,6 +147,7 @@ sr_debug_gather_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d
   const int p = blockIdx.x;
   if (p * SR_PAGE_ROWS >= R) return;
   const int slot = s.req_slot0[i] + p;
+  if (!sr_check_slot(s, slot) || !sr_check_page(s, s.slot_page[slot])) return;
   const int rows = s.slot_rows[slot];
   const char* src = pool.base + (int64_t)s.slot_page[slot] * pool.page_stride + (int64_t)pool_layer * pool.layer_stride;
   const int64_t row0 = (int64_t)s.req_row0[i] + (int64_t)p * SR_PAGE_ROWS;

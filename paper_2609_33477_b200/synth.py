@@ -96,6 +96,8 @@ SPECS = {
                                n_requests=2, replay=("list", (70, 129))),
     "geom_96_192": WorkloadSpec(name="geom_96_192", n_layers=1, d_model=256, n_k_heads=3, n_v_heads=3, d_k=96, d_v=192,
                                 n_requests=3, replay=("list", (200, 64, 321))),
+    # many layers, a small batch: the layers of one call run side by side
+    "layers_small": _spec("layers_small", 9, 512, 4, 128, 3, ("list", (130, 64, 257)), layer_mask="all"),
     # the per-head-decay family (no erase)
     "decay_only_small": _spec("decay_only_small", 2, 512, 4, 128, 4, ("list", (130, 64, 257, 5)), recurrence="decay_only"),
     "decay_only_d64": _spec("decay_only_d64", 1, 256, 2, 64, 3, ("list", (70, 128, 3)), recurrence="decay_only"),
@@ -112,6 +114,20 @@ SPECS = {
     "cfg4_slice": _spec("cfg4_slice", 1, 5120, 32, 128, 4, ("fixed", 8192),
                         weight_format="e4m3_block128", decay_scale=0.03),
 }
+# The head geometry of the paper's three models (Appendix A table) at their own d_model, two layers, 8 requests of
+# 2048 rows: bench lines for the widths the five configurations do not cover.
+SPECS["model_4b"] = WorkloadSpec(name="model_4b", n_layers=2, d_model=2560, n_k_heads=16, n_v_heads=32, d_k=128,
+                                 d_v=128, n_requests=8, replay=("fixed", 2048))
+SPECS["model_27b"] = WorkloadSpec(name="model_27b", n_layers=2, d_model=5120, n_k_heads=16, n_v_heads=48, d_k=128,
+                                  d_v=128, n_requests=8, replay=("fixed", 2048))
+SPECS["model_7b_96_192"] = WorkloadSpec(name="model_7b_96_192", n_layers=2, d_model=3840, n_k_heads=30, n_v_heads=30,
+                                        d_k=96, d_v=192, n_requests=8, replay=("fixed", 2048))
+# The paper's own operating point (Section 6: at most 512 anchors per hit on the 4B model, 4096 packed anchors per
+# batch): one hit, and eight simultaneous hits, all 24 linear layers of the 4B geometry.
+SPECS["hit_512"] = WorkloadSpec(name="hit_512", n_layers=24, d_model=2560, n_k_heads=16, n_v_heads=32, d_k=128,
+                                d_v=128, n_requests=1, replay=("fixed", 512))
+SPECS["hits8_512"] = WorkloadSpec(name="hits8_512", n_layers=24, d_model=2560, n_k_heads=16, n_v_heads=32, d_k=128,
+                                  d_v=128, n_requests=8, replay=("fixed", 512))
 for _r in (1024, 2048, 4096):
     SPECS[f"cfg4_R{_r}"] = dataclasses.replace(SPECS["cfg4"], name=f"cfg4_R{_r}", replay=("fixed", _r))
 

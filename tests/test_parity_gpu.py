@@ -291,6 +291,10 @@ def test_host_buffer_entry_with_a_row_major_pool_goes_up_in_one_piece():
     (B.SR_DEBUG_DOT_CONV_STATE, "ragged_small"),  # conv state by per-channel dot products
     (B.SR_DEBUG_DOT_CONV_STATE, "fp8_small"),
     (B.SR_DEBUG_SINGLE_CTA_MMA, "cfg1_narrow"),   # one-CTA form of the fused projection
+    (B.SR_DEBUG_CHECK_BOUNDS, "ragged_small"),    # device-side range checks on: same results, no flag raised
+    (B.SR_DEBUG_CHECK_BOUNDS, "trunks_small"),
+    (B.SR_DEBUG_CHECK_BOUNDS, "geom_96_192"),
+    (B.SR_DEBUG_CHECK_BOUNDS | B.SR_DEBUG_DOT_CONV_STATE, "fp8_small"),
 ])
 def test_second_forms_match_oracle(flag, name):
     wl, rep = _run(name, debug_flags=flag)
@@ -298,6 +302,38 @@ def test_second_forms_match_oracle(flag, name):
     for i in range(wl.spec.n_requests):
         for l in _active(wl):
             U.check_request_layer(rep, wl, i, l)
+
+
+# ----------------------------------------------------- layers of one call side by side
+
+def test_layers_run_side_by_side_with_the_same_bits_as_one_after_the_other():
+    """A small batch with nine rebuilt layers: with the recommended workspace the call spreads the layers over
+    four streams of the context, with the minimum workspace it runs them in order.  Same bits either way, and
+    both match the oracle."""
+    wl = synth.build_workload("layers_small", device=DEV)
+    wide = B.Replayer(wl)
+    narrow = B.Replayer(wl, min_workspace=True)
+    assert wide.workspace_bytes > narrow.workspace_bytes
+    for rep in (wide, narrow):
+        for _ in range(2):
+            rep.out_ssm.fill_(float("nan"))
+            rep.replay_states()
+            torch.cuda.synchronize()
+            assert rep.device_status() == 0
+    assert torch.equal(wide.out_ssm, narrow.out_ssm) and torch.equal(wide.out_conv, narrow.out_conv)
+    for l in (0, 4, 8):
+        for i in range(wl.spec.n_requests):
+            U.check_request_layer(wide, wl, i, l)
+    # and inside a captured graph: the side streams fork from and join the capturing stream
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        wide.replay_states(torch.cuda.current_stream())
+    wide.out_ssm.zero_()
+    wide.out_conv.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(wide.out_ssm, narrow.out_ssm) and torch.equal(wide.out_conv, narrow.out_conv)
 
 
 # ----------------------------------------------------- a bounded in-kernel wait that runs out
