@@ -42,8 +42,9 @@ orthonormal keys, single-row and overwrite cases (the single-row closed form and
 test also at H_v != H_k and d_k != d_v, which pin the q | k | v channel split), continuation from a cut (of the
 recurrence, of the convolution with its history, and of a whole layer replayed in two
 pieces against one pass), the contraction bound of the replay error, library convolution /
-activation routines, all 256 e4m3 codes, the state sizes printed in the paper's
-Appendix A table, and a write / gather round trip.
+activation routines, all 256 e4m3 codes, the e4m3 activation quantiser (codes and scales bit for bit
+against a library cast, every representable value as a fixed point, ties and saturation, the half-step
+error bound), the state sizes printed in the paper's Appendix A table, and a write / gather round trip.
 """
 
 from __future__ import annotations
@@ -91,6 +92,44 @@ def dequant_block_scaled(codes, scales, block: int = 128) -> np.ndarray:
     rows = np.arange(C) // block
     cols = np.arange(d) // block
     return w * np.asarray(scales, dtype=np.float64)[rows[:, None], cols[None, :]]
+
+
+def f32_to_e4m3_codes(y) -> np.ndarray:
+    """fp32 values -> e4m3 codes, round to nearest even, magnitudes above 448 saturate to 448 (never NaN)."""
+    y = np.asarray(y, dtype=np.float32).astype(np.float64)
+    sign = np.where(np.signbit(y), 0x80, 0).astype(np.int64)
+    a = np.minimum(np.abs(y), 448.0)
+    m, e = np.frexp(a)                                   # a = m * 2^e, m in [0.5, 1)
+    e = e - 1                                            # a = (2m) * 2^e, 2m in [1, 2)
+    sub = a < 2.0 ** -6                                  # below the smallest normal: steps of 2^-9
+    q_sub = np.rint(a / 2.0 ** -9).astype(np.int64)      # 0..8 (8 = the smallest normal, code 0x08)
+    frac = np.rint((2.0 * m - 1.0) * 8.0).astype(np.int64)      # 0..8, ties to even
+    e_n = np.where(frac == 8, e + 1, e)
+    frac = np.where(frac == 8, 0, frac)
+    q_norm = ((e_n + 7) << 3) | frac
+    code = np.where(sub, q_sub, q_norm)
+    return (sign | code).astype(np.uint8)
+
+
+def quantise_e4m3_1x128(X, group: int = 128):
+    """Activation quantiser of the W8A8 variant: each row is cut into groups of 128 consecutive channels; per
+    group s = max(amax, 1e-10) / 448 and code = e4m3(x / s), both in fp32 with IEEE division and
+    round-to-nearest-even.  X [R, d] (values exactly representable in fp32) -> (codes uint8 [R, d], scales
+    float32 [R, d / group])."""
+    X32 = np.asarray(X, dtype=np.float32)
+    R, d = X32.shape
+    g = X32.reshape(R, d // group, group)
+    amax = np.max(np.abs(g), axis=-1)
+    scale = (np.maximum(amax, np.float32(1e-10)) / np.float32(448.0)).astype(np.float32)
+    codes = f32_to_e4m3_codes((g / scale[:, :, None]).astype(np.float32)).reshape(R, d)
+    return codes, scale
+
+
+def dequantise_1x128(codes, scales, group: int = 128) -> np.ndarray:
+    """decode(code) * scale of its (row, group), exact in fp64."""
+    R, d = codes.shape
+    return (e4m3_decode(codes).reshape(R, d // group, group) *
+            np.asarray(scales, dtype=np.float64)[:, :, None]).reshape(R, d)
 
 
 # ---------------------------------------------------------------------------------------
@@ -240,13 +279,19 @@ def gated_delta_recurrence(k_hat, v, alpha, beta, S0=None, erase: bool = True) -
 # the whole path for one (request, layer)
 
 def replay_layer(X, w_qkv, w_ab, conv_w, decay_scale, dt_bias, *, n_k_heads, n_v_heads, d_k, d_v,
-                 eps: float = 1e-6, activation: str = "silu", S0=None, conv_state_bits=None, erase: bool = True):
+                 eps: float = 1e-6, activation: str = "silu", S0=None, conv_state_bits=None, erase: bool = True,
+                 act_quant: str = "none"):
     """Anchor rows X [R, d] (fp64) -> (S fp32 [H_v, d_k, d_v], conv state uint16 [C, w-1]).
 
     Replay from a zero state (Eq. 4, S_0 = 0) by default.  With `S0` ([H_v, d_k, d_v]) and `conv_state_bits`
     ([C, w-1] uint16, the layout this function returns) the same rows continue an earlier state instead: the
     recurrence starts from S0 (Eq. 5 with a non-zero carried term) and the convolution sees the stored inputs
-    as the rows before row 0 (Appendix A: the conv state is the last w-1 inputs of each channel)."""
+    as the rows before row 0 (Appendix A: the conv state is the last w-1 inputs of each channel).
+
+    `act_quant="e4m3_1x128"` is the W8A8 variant of the block-scaled projection (Section 7.1 runs the 27B model
+    with FP8 weights): the rows that enter the q | k | v projection are first quantised to e4m3 with one scale
+    per row and 128 channels and the projection uses the dequantised values.  The gate projection, whose weights
+    stay bf16, keeps the unquantised rows."""
     conv_w = np.asarray(conv_w, dtype=np.float64)
     width = conv_w.shape[1]
     C = 2 * n_k_heads * d_k + n_v_heads * d_v
@@ -258,6 +303,10 @@ def replay_layer(X, w_qkv, w_ab, conv_w, decay_scale, dt_bias, *, n_k_heads, n_v
                     else np.array(conv_state_bits, dtype=np.uint16))
         return S_out, tail_out
     Z, G = in_projection(X, w_qkv, w_ab)
+    if act_quant == "e4m3_1x128":
+        Z, _ = in_projection(dequantise_1x128(*quantise_e4m3_1x128(X)), w_qkv, w_ab)
+    elif act_quant != "none":
+        raise ValueError(act_quant)
     tail = conv_tail_bits(Z, width, history)
     Y = causal_conv_silu(Z, conv_w, activation, history)
     _q, k, v = split_qkv(Y, n_k_heads, n_v_heads, d_k, d_v)
@@ -279,7 +328,7 @@ def layer_weights_f64(arrays: dict):
 
 def replay_request_layer(pool, pages, n_rows, pool_layer, arrays: dict, *, n_k_heads, n_v_heads, d_k, d_v,
                          eps: float = 1e-6, activation: str = "silu", S0=None, conv_state_bits=None,
-                         erase: bool = True):
+                         erase: bool = True, act_quant: str = "none"):
     """Gather + replay for one (request, layer) from raw storage."""
     w_qkv, w_ab, conv_w, c, delta = layer_weights_f64(arrays)
     X = gather_anchor_rows(pool, pages, n_rows, pool_layer)
@@ -287,7 +336,7 @@ def replay_request_layer(pool, pages, n_rows, pool_layer, arrays: dict, *, n_k_h
         X = np.zeros((0, w_qkv.shape[1]))
     return replay_layer(X, w_qkv, w_ab, conv_w, c, delta, n_k_heads=n_k_heads, n_v_heads=n_v_heads,
                         d_k=d_k, d_v=d_v, eps=eps, activation=activation, S0=S0, conv_state_bits=conv_state_bits,
-                        erase=erase)
+                        erase=erase, act_quant=act_quant)
 
 
 # ---------------------------------------------------------------------------------------

@@ -289,7 +289,7 @@ sr_hist_gather_kernel(SrSched s, const char* __restrict__ in_layer, int64_t slot
 // The GEMM reads every weight once per 64 tail rows but walks d_model serially in one CTA per 64 channels; below
 // GEMM_MIN_REQUESTS requests the dot-product kernel (a warp per channel and request, thousands of short chains)
 // finishes sooner.
-constexpr int GEMM_MIN_REQUESTS = 16;
+constexpr int GEMM_MIN_REQUESTS = 4;
 
 static bool conv_tail_gemm_fits(const sr_ctx* ctx, int n_requests) {
   const bool fp8 = ctx->desc.weight_format == SR_W_E4M3_BLOCK128;

@@ -61,6 +61,83 @@ def test_e4m3_decode_all_256_codes_against_torch_and_closed_form():
     assert ours[0x38] == 1.0 and ours[0xB8] == -1.0 and np.isnan(ours[0x7F]) and np.isnan(ours[0xFF])
 
 
+def test_e4m3_rounding_every_code_is_a_fixed_point_and_ties_go_to_even():
+    codes = np.array([c for c in range(256) if (c & 0x7F) != 0x7F], dtype=np.uint8)
+    vals = orc.e4m3_decode(codes)
+    back = orc.f32_to_e4m3_codes(vals.astype(np.float32))
+    assert np.array_equal(back & 0x7F, codes & 0x7F)                       # every value maps to its own code
+    assert np.array_equal(back[vals != 0] & 0x80, codes[vals != 0] & 0x80)
+    # midpoints between neighbours go to the even code; a hair to either side goes to the nearer one
+    pos = np.sort(vals[codes < 0x80])                                      # the non-negative values, +0 once
+    lo, hi = pos[:-1], pos[1:]
+    mid = ((lo + hi) / 2).astype(np.float32)                              # exact in fp32
+    c_lo, c_hi = orc.f32_to_e4m3_codes(lo.astype(np.float32)), orc.f32_to_e4m3_codes(hi.astype(np.float32))
+    want = np.where(c_lo % 2 == 0, c_lo, c_hi)
+    assert np.array_equal(orc.f32_to_e4m3_codes(mid), want)
+    assert np.array_equal(orc.f32_to_e4m3_codes(np.nextafter(mid, np.float32(0))), c_lo)
+    assert np.array_equal(orc.f32_to_e4m3_codes(np.nextafter(mid, np.float32(1e9))), c_hi)
+    # saturation instead of NaN, signs kept
+    assert orc.f32_to_e4m3_codes(np.float32([449.0, 1e9, -1e9, 464.0, -0.0])).tolist() == [0x7E, 0x7E, 0xFE, 0x7E, 0x80]
+
+
+def test_e4m3_rounding_matches_the_library_cast_inside_the_range():
+    r = _rng(61)
+    y = np.concatenate([r.standard_normal(50000) * 10.0 ** r.uniform(-4, 2.6, 50000), r.uniform(-448, 448, 20000)])
+    y = y[np.abs(y) <= 448].astype(np.float32)
+    lib = torch.from_numpy(y).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(orc.f32_to_e4m3_codes(y), lib)
+
+
+def test_activation_quantiser_scales_codes_and_error_bound():
+    r = _rng(62)
+    X = torch.from_numpy(r.standard_normal((9, 384)) * 10.0 ** r.uniform(-3, 3, (9, 1))).to(torch.bfloat16)
+    X[3, 128:256] = 0                                           # an all-zero group: scale floor, codes zero
+    Xf = X.float().numpy()
+    codes, scales = orc.quantise_e4m3_1x128(Xf)
+    assert codes.shape == (9, 384) and scales.shape == (9, 3) and scales.dtype == np.float32
+    # the same arithmetic through torch: fp32 amax, fp32 divisions, library cast
+    g = X.float().reshape(9, 3, 128)
+    s_t = torch.clamp(g.abs().amax(-1), min=1e-10) / 448.0
+    c_t = (g / s_t[:, :, None]).to(torch.float8_e4m3fn).view(torch.uint8).reshape(9, 384).numpy()
+    assert np.array_equal(scales, s_t.numpy()) and np.array_equal(codes, c_t)
+    assert not codes[3, 128:256].any() and scales[3, 1] == np.float32(1e-10) / np.float32(448)
+    # the largest magnitude of every group lands on +-448, and nothing is off by more than half a step of its binade
+    deq = orc.dequantise_1x128(codes, scales)
+    y = Xf.astype(np.float64).reshape(9, 3, 128) / scales.astype(np.float64)[:, :, None]
+    step = np.maximum(2.0 ** (np.floor(np.log2(np.maximum(np.abs(y), 2.0 ** -6))) - 3), 2.0 ** -9)
+    err = np.abs(deq.reshape(9, 3, 128) / scales.astype(np.float64)[:, :, None] - y)
+    assert np.all(err <= step / 2 * (1 + 1e-6) + 448 * 2.0 ** -23)
+    nz = [(i, j) for i in range(9) for j in range(3) if not (i == 3 and j == 1)]
+    assert all(np.abs(orc.e4m3_decode(codes.reshape(9, 3, 128)[i, j])).max() == 448.0 for i, j in nz)
+
+
+def test_w8a8_layer_is_the_layer_on_dequantised_rows_with_exact_gates():
+    """act_quant: the q | k | v projection sees decode(code) * scale, the gate projection the original rows."""
+    r = _rng(63)
+    R, d, H, dk = 11, 256, 2, 4
+    C = 3 * H * dk
+    X = torch.from_numpy(r.standard_normal((R, d))).to(torch.bfloat16).double().numpy()
+    W = r.standard_normal((C, d)) / math.sqrt(d)
+    Wab = r.standard_normal((2 * H, d)) / math.sqrt(d)
+    cw = r.standard_normal((C, 4)) / 2
+    c, delta = np.array([0.1, 0.2]), np.zeros(2)
+    kw = dict(n_k_heads=H, n_v_heads=H, d_k=dk, d_v=dk)
+    S_q, tail_q = orc.replay_layer(X, W, Wab, cw, c, delta, act_quant="e4m3_1x128", **kw)
+    Xd = orc.dequantise_1x128(*orc.quantise_e4m3_1x128(X))
+    assert 1e-3 < np.abs(Xd - X).max() / np.abs(X).max() < 0.07          # really quantised: e4m3 keeps 4 bits
+    # the same thing spelled out with the step functions: Z from the dequantised rows, G from the original ones
+    Z = Xd @ W.T
+    G = X @ Wab.T
+    Y = orc.causal_conv_silu(Z, cw)
+    _, k, v = orc.split_qkv(Y, H, H, dk, dk)
+    alpha, beta = orc.gates(G, c, delta)
+    S_want = orc.gated_delta_recurrence(orc.l2_normalise(k), v, alpha, beta)
+    assert np.allclose(S_q, S_want.astype(np.float32), rtol=1e-6, atol=1e-9)
+    assert np.array_equal(tail_q, orc.conv_tail_bits(Z, 4))
+    S_plain, _ = orc.replay_layer(X, W, Wab, cw, c, delta, **kw)
+    assert not np.allclose(S_q, S_plain, rtol=1e-3)                        # and it differs from the exact-activation layer
+
+
 def test_block_scaled_dequant_brute_force():
     r = _rng(2)
     C, d = 200, 384
