@@ -70,6 +70,16 @@ typedef enum sr_status {
 
 enum { SR_W_BF16 = 0, SR_W_E4M3_BLOCK128 = 1 };   /* sr_model_desc.weight_format   */
 enum { SR_CONV_SILU = 0, SR_CONV_IDENTITY = 1 };  /* sr_model_desc.conv_activation */
+/* sr_model_desc.act_quant: what the q | k | v projection multiplies the e4m3 weights with (Section 7.1 serves the
+ * 27B model with FP8 weights).  NONE (default): the bf16 anchors as they are (W8A16): the result is the exact
+ * product up to fp32 summation and one 16-bit rounding of each weight.  E4M3_1X128 (W8A8, weight_format
+ * SR_W_E4M3_BLOCK128 only): each anchor row is quantised on the fly, 128 channels at a time, s = max(amax, 1e-10)/448,
+ * code = e4m3(x / s) (fp32, IEEE division, round to nearest even, saturating), and the products run on the 8-bit
+ * tensor-core path at twice the 16-bit rate; a 128-deep partial sum enters the result as
+ * weight scale x activation scale x partial sum in fp32.  The gate projection (bf16 weights) keeps the bf16 rows.
+ * W8A8 changes the VALUE computed (e4m3 keeps 4 significant bits of each activation): it is its own variant with
+ * its own reference result, not an approximation of NONE held to the same tolerance. */
+enum { SR_AQ_NONE = 0, SR_AQ_E4M3_1X128 = 1 };
 /* sr_model_desc.recurrence: the transition A_t of Eq. 4 (Section 2.1 names both families).
  * GATED_DELTA: A_t(S) = alpha_t (I - beta_t k_t k_t^T) S.  DECAY_ONLY: A_t(S) = alpha_t S (per-head decay, no
  * erase).  The write B_t = beta_t k_t v_t^T and everything before the recurrence are the same. */
@@ -102,6 +112,7 @@ typedef struct sr_model_desc {
   float l2_eps;            /* epsilon inside the key normalisation (1e-6)               */
   int32_t recurrence;      /* SR_REC_* (0 = gated delta rule)                           */
   uint32_t debug_flags;    /* SR_DEBUG_* test and diagnostic switches; 0 in production  */
+  int32_t act_quant;       /* SR_AQ_* (0 = none)                                        */
 } sr_model_desc;
 
 /* One layer's parameters: HOST struct holding DEVICE pointers.  The array handed to
@@ -336,6 +347,16 @@ int sr_debug_gather(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table
                     const int32_t* replay_lens, int32_t layer, void* out_rows,
                     int64_t out_capacity_rows, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * W8A8 only (act_quant = SR_AQ_E4M3_1X128): materialises what the activation quantiser produces for one layer, for
+ * the bit-exact check of codes and scales: out_codes DEVICE uint8 [sum of replay_lens][d_model], out_scales DEVICE
+ * fp32 [sum of replay_lens][d_model / 128], requests packed in order like sr_debug_gather.  A test and diagnostic
+ * entry; the replay call keeps the codes in its workspace.
+ */
+int sr_debug_quantise(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* table, const int32_t* replay_lens,
+                      int32_t layer, void* out_codes, float* out_scales, int64_t out_capacity_rows, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
 /* Waits for `stream` and returns the device status word the last call on this
  * workspace left (SR_DEV_* bits).  Synchronising; for tests and diagnostics. */
 int sr_device_status(sr_ctx* ctx, const void* workspace, void* stream, uint32_t* out_flags);
@@ -352,7 +373,7 @@ enum {
   SR_KERNEL_SCAN = 3,       /* conv + SiLU + norm + gates + gated-delta state scan    */
   SR_KERNEL_WEIGHT_DECODE = 4, /* e4m3 weights only: codes -> 16-bit weights before the projection */
   SR_KERNEL_CHUNK_LOCAL = 5,   /* gates, K K^T and the chunk inverse for all chunks at once (then SCAN is the chain) */
-  SR_KERNEL_ANCHOR_STAGE = 6,  /* e4m3 weights only: the layer's anchors copied to fp16 in slot order */
+  SR_KERNEL_ANCHOR_STAGE = 6,  /* e4m3 weights only: the layer's anchors copied to fp16 (W8A16) or quantised to e4m3 (W8A8), slot order */
   SR_KERNEL_KINDS = 7
 };
 

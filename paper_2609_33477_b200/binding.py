@@ -23,6 +23,7 @@ SR_DEV_BAD_REPLAY_LEN, SR_DEV_BAD_PAGE_ID, SR_DEV_BAD_SLOT, SR_DEV_ROWS_OVERFLOW
 SR_W_BF16, SR_W_E4M3_BLOCK128 = 0, 1
 SR_CONV_SILU, SR_CONV_IDENTITY = 0, 1
 SR_REC_GATED_DELTA, SR_REC_DECAY_ONLY = 0, 1
+SR_AQ_NONE, SR_AQ_E4M3_1X128 = 0, 1
 SR_DEV_BOUNDS_CHECK = 32
 SR_DEBUG_DOT_CONV_STATE, SR_DEBUG_SINGLE_CTA_MMA, SR_DEBUG_FP8_EXACT, SR_DEBUG_CHECK_BOUNDS, SR_DEBUG_EXPIRE_WAIT = 1, 2, 4, 8, 16
 
@@ -31,6 +32,7 @@ EXPORTS = (
     "sr_conv_bytes_per_layer", "sr_workspace_bytes", "sr_replay_states", "sr_replay_states_host",
     "sr_debug_gather", "sr_device_status", "sr_last_launch_count", "sr_profile_enable", "sr_profile_read",
     "sr_replay_states_noalloc", "sr_replay_states_from", "sr_anchor_write", "sr_workspace_bytes_min",
+    "sr_debug_quantise",
 )
 SR_NOALLOC_SCRATCH_BYTES = 128 * 1024 * 1024
 SR_KERNEL_SCHEDULE, SR_KERNEL_PROJECTION, SR_KERNEL_CONV_TAIL, SR_KERNEL_SCAN = 0, 1, 2, 3
@@ -42,7 +44,7 @@ class sr_model_desc(C.Structure):
                 ("n_v_heads", C.c_int32), ("d_k", C.c_int32), ("d_v", C.c_int32),
                 ("conv_width", C.c_int32), ("page_rows", C.c_int32), ("weight_format", C.c_int32),
                 ("conv_activation", C.c_int32), ("l2_eps", C.c_float), ("recurrence", C.c_int32),
-                ("debug_flags", C.c_uint32)]
+                ("debug_flags", C.c_uint32), ("act_quant", C.c_int32)]
 
 
 class sr_layer_weights(C.Structure):
@@ -110,6 +112,9 @@ def load() -> C.CDLL:
         C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     lib.sr_debug_gather.argtypes = [
         C.c_void_p, C.POINTER(sr_anchor_pool), C.POINTER(sr_page_table), C.c_void_p, C.c_int32, C.c_void_p,
+        C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sr_debug_quantise.argtypes = [
+        C.c_void_p, C.POINTER(sr_anchor_pool), C.POINTER(sr_page_table), C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
         C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sr_device_status.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_uint32)]
     lib.sr_last_launch_count.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
@@ -210,6 +215,12 @@ def sr_debug_gather(ctx, pool, table, replay_lens_ptr, layer, out_rows_ptr, capa
                                   capacity_rows, workspace_ptr, workspace_bytes, stream_ptr)
 
 
+def sr_debug_quantise(ctx, pool, table, replay_lens_ptr, layer, out_codes_ptr, out_scales_ptr, capacity_rows,
+                      workspace_ptr, workspace_bytes, stream_ptr) -> int:
+    return load().sr_debug_quantise(ctx, C.byref(pool), C.byref(table), replay_lens_ptr, layer, out_codes_ptr,
+                                    out_scales_ptr, capacity_rows, workspace_ptr, workspace_bytes, stream_ptr)
+
+
 def sr_device_status(ctx, workspace_ptr, stream_ptr) -> int:
     v = C.c_uint32()
     _check(load().sr_device_status(ctx, workspace_ptr, stream_ptr, C.byref(v)), "sr_device_status")
@@ -239,7 +250,7 @@ def model_desc(spec, conv_activation: int = SR_CONV_SILU, l2_eps: float = 1e-6, 
     return sr_model_desc(spec.n_layers, spec.d_model, spec.n_k_heads, spec.n_v_heads, spec.d_k, spec.d_v,
                          spec.conv_width, 64, fmt, conv_activation, l2_eps,
                          SR_REC_DECAY_ONLY if getattr(spec, "recurrence", "gated_delta") == "decay_only" else SR_REC_GATED_DELTA,
-                         debug_flags)
+                         debug_flags, SR_AQ_E4M3_1X128 if getattr(spec, "act_quant", "none") == "e4m3_1x128" else SR_AQ_NONE)
 
 
 class Replayer:
@@ -367,6 +378,16 @@ class Replayer:
                              rows, self._ws_ptr, self.workspace_bytes, self._stream_ptr(stream))
         _check(st, "sr_debug_gather")
         return out
+
+    def debug_quantise(self, layer: int, stream=None):
+        """W8A8 contexts: the activation codes [rows, d] (uint8) and scales [rows, d / 128] (fp32) of one layer."""
+        rows = max(1, int(self.table.max_total_rows))
+        codes = torch.zeros((rows, self.spec.d_model), dtype=torch.uint8, device=self.device)
+        scales = torch.zeros((rows, self.spec.d_model // 128), dtype=torch.float32, device=self.device)
+        st = sr_debug_quantise(self.ctx, self.pool, self.table, self.wl.replay_lens.data_ptr(), layer, codes.data_ptr(),
+                               scales.data_ptr(), rows, self._ws_ptr, self.workspace_bytes, self._stream_ptr(stream))
+        _check(st, "sr_debug_quantise")
+        return codes, scales
 
     def device_status(self, stream=None) -> int:
         return sr_device_status(self.ctx, self._ws_ptr, self._stream_ptr(stream))

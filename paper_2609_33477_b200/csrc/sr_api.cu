@@ -133,6 +133,8 @@ int sr_create(const sr_model_desc* d, sr_ctx** out_ctx) {
   if (d->weight_format != SR_W_BF16 && d->weight_format != SR_W_E4M3_BLOCK128) return SR_ERR_INVALID_ARG;
   if (d->conv_activation != SR_CONV_SILU && d->conv_activation != SR_CONV_IDENTITY) return SR_ERR_INVALID_ARG;
   if (d->recurrence != SR_REC_GATED_DELTA && d->recurrence != SR_REC_DECAY_ONLY) return SR_ERR_INVALID_ARG;
+  if (d->act_quant != SR_AQ_NONE && d->act_quant != SR_AQ_E4M3_1X128) return SR_ERR_INVALID_ARG;
+  if (d->act_quant == SR_AQ_E4M3_1X128 && d->weight_format != SR_W_E4M3_BLOCK128) return SR_ERR_INVALID_ARG;
   if (!(d->l2_eps >= 0.f)) return SR_ERR_INVALID_ARG;
   if (d->conv_width < 2 || d->page_rows <= 0 || d->n_v_heads % d->n_k_heads != 0) return SR_ERR_INVALID_ARG;
   sr_ctx* c = new (std::nothrow) sr_ctx;
@@ -155,11 +157,14 @@ int sr_create(const sr_model_desc* d, sr_ctx** out_ctx) {
   c->kernels_cover = d->conv_width == SR_CONV_W && d->page_rows == SR_PAGE_ROWS && sr_proj_fused_supported(c) &&
                      sr_chunk_local_supported(d->d_k, d->d_v) && sr_scan_chain_supported(d->d_k, d->d_v);
   const bool e4m3 = d->weight_format == SR_W_E4M3_BLOCK128;
+  c->w8a8 = e4m3 && d->act_quant == SR_AQ_E4M3_1X128;
+  // 8-bit operands: channel tiles inside the scale blocks, and the batched conv-state kernel's tiling
+  if (c->w8a8 && !(sr_proj_fused_exact_fp8_supported(c) && c->conv_ch % 64 == 0 && c->n_gate <= 256)) c->kernels_cover = false;
   // block-scaled weights: fp16 staging by default; fp32 promotion of bare-code partial sums on request, where the
   // channel tiles line up with the scale blocks
-  c->fp16_stage = c->kernels_cover && e4m3 &&
+  c->fp16_stage = c->kernels_cover && e4m3 && !c->w8a8 &&
                   !((d->debug_flags & SR_DEBUG_FP8_EXACT) && sr_proj_fused_exact_fp8_supported(c));
-  if (c->kernels_cover && e4m3)
+  if (c->kernels_cover && e4m3 && !c->w8a8)
     c->wdec_bytes = (size_t)(c->n_k + c->n_v + (c->fp16_stage ? c->n_gate : 0)) * d->d_model * 2;
   *out_ctx = c;
   return SR_OK;
@@ -332,6 +337,8 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
     fused.hist = nullptr;
     fused.in_ssm_layer = nullptr;
     fused.in_ssm_slot_stride = 0;
+    fused.x8 = ctx->w8a8 ? (const uint8_t*)(base + lay.off_x16) : nullptr;
+    fused.sx = ctx->w8a8 ? (const float*)(base + lay.off_sx) : nullptr;
     fused.x16 = ctx->fp16_stage ? (const __half*)(base + lay.off_x16) : nullptr;
     fused.w16 = ctx->fp16_stage ? (const __half*)(base + lay.off_wdec) : nullptr;
     const int pl = pool->layer_to_pool[l];
@@ -361,12 +368,17 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
         }
         LaunchScope scope(ctx, ls, SR_KERNEL_ANCHOR_STAGE);
         if (sr_launch_stage_anchors_fp16(ctx, sched, pv, pl, (__half*)(base + lay.off_x16), ls) != cudaSuccess) break;
+      } else if (ctx->w8a8) {
+        LaunchScope scope(ctx, ls, SR_KERNEL_ANCHOR_STAGE);
+        if (sr_launch_quant_anchors_e4m3(ctx, sched, pv, pl, (uint8_t*)(base + lay.off_x16), (float*)(base + lay.off_sx), ls) !=
+            cudaSuccess)
+          break;
       } else if (ctx->wdec_bytes) {
         LaunchScope scope(ctx, ls, SR_KERNEL_WEIGHT_DECODE);
         if (sr_launch_weight_decode(ctx, weights[l], wdec, ls) != cudaSuccess) break;
       }
       {
-        LaunchScope scope(ctx, ls, SR_KERNEL_PROJECTION);
+        LaunchScope scope(ctx, ls, SR_KERNEL_PROJECTION, ctx->w8a8 ? 2 : 1);
         if (sr_launch_proj_fused(ctx, sched, *pool, pl, weights[l], ctx->wdec_bytes ? wdec : nullptr, fused, sm_count,
                                  ls) != cudaSuccess)
           break;
@@ -638,6 +650,38 @@ int sr_debug_gather(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table
                              out_rows, out_capacity_rows, stream) != cudaSuccess)
     return SR_ERR_CUDA;
   ctx->last_launches = 2;
+  return SR_OK;
+}
+
+int sr_debug_quantise(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* table, const int32_t* replay_lens,
+                      int32_t layer, void* out_codes, float* out_scales, int64_t out_capacity_rows, void* workspace,
+                      size_t workspace_bytes, void* stream_) {
+  int st = check_batch(ctx, table);
+  if (st != SR_OK) return st;
+  if (!ctx->w8a8) return SR_ERR_UNSUPPORTED_SHAPE;
+  if (!replay_lens || !out_codes || !out_scales || !table->pages || out_capacity_rows < 0) return SR_ERR_INVALID_ARG;
+  st = check_pool(ctx, pool);
+  if (st != SR_OK) return st;
+  if (layer < 0 || layer >= ctx->desc.n_layers || pool->layer_to_pool[layer] < 0) return SR_ERR_INVALID_ARG;
+  if (!aligned(out_codes, 16) || !aligned(out_scales, 4)) return SR_ERR_INVALID_ARG;
+  const SrWorkspace lay = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows);
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < lay.total) return SR_ERR_WORKSPACE;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  ctx->last_launches = 0;
+  if (table->n_requests == 0 || table->max_pages == 0) return SR_OK;
+  SrSched sched = sr_sched_view(workspace, lay, table->n_requests);
+  sched.n_phys_pages = pool->n_phys_pages;
+  ctx->ev_used = 0;
+  ctx->ev_kind.clear();
+  uint8_t* x8 = (uint8_t*)workspace + lay.off_x16;
+  float* sx = (float*)((char*)workspace + lay.off_sx);
+  if (sr_launch_schedule(sched, table->pages, table->state_slots, replay_lens, table->max_pages, table->max_replay_len,
+                         table->max_total_rows, pool->n_phys_pages, table->n_state_slots, stream) != cudaSuccess ||
+      sr_launch_quant_anchors_e4m3(ctx, sched, pool_view(pool), pool->layer_to_pool[layer], x8, sx, stream) != cudaSuccess ||
+      sr_launch_pack_quantised(ctx, sched, table->max_pages, x8, sx, out_codes, out_scales, out_capacity_rows, stream) !=
+          cudaSuccess)
+    return SR_ERR_CUDA;
+  ctx->last_launches = 3;
   return SR_OK;
 }
 

@@ -31,6 +31,7 @@ struct sr_ctx {
                        // once per layer, then the same tensor-core kernel as for bf16 weights (SR_DEBUG_FP8_EXACT
                        // selects fp32 promotion of bare-code partial sums instead)
   uint32_t debug_flags;  // desc.debug_flags (SR_DEBUG_*)
+  bool w8a8;             // e4m3 weights x on-the-fly e4m3 activations on the 8-bit tensor-core path
   // optional per-kernel timing (sr_profile_*): events bracketing every launch of the last call
   bool profiling;
   std::vector<cudaEvent_t> ev_pool;   // created on demand, reused, destroyed with the context
@@ -78,7 +79,9 @@ struct SrWorkspace {
                          // kernel to the chain kernel
   size_t off_wdec;       // [n_k + n_v (+ 2 H_v)][d_model] 16-bit decoded weights of the current layer (0 bytes for bf16 weights)
   size_t off_hist;       // bf16 [n_requests][C][w-1] conv state each request continues from (current layer)
-  size_t off_x16;        // fp16 staging: half [max_slots][64][d_model] anchors of the current layer, slot order
+  size_t off_x16;        // fp16 staging: half [max_slots][64][d_model] anchors of the current layer, slot order;
+                         // W8A8: uint8 [max_slots][64][d_model] activation codes
+  size_t off_sx;         // W8A8: float [max_slots][d_model / 128][64] activation scales
   size_t lane_bytes;     // size of one lane's block of hand-over buffers (off_kv16 .. end)
   int lanes;             // lane blocks in `total`
   size_t total;
@@ -116,8 +119,10 @@ static inline SrWorkspace sr_workspace_layout(const sr_ctx* ctx, int32_t n_reque
   w.off_split = at;     at = sr_align256(at + sr_scan_split_bytes(ctx, w.max_slots));
   w.off_wdec = at;      at = sr_align256(at + ctx->wdec_bytes);
   w.off_hist = at;      at = sr_align256(at + sizeof(uint16_t) * (size_t)n_requests * ctx->conv_ch * (SR_CONV_W - 1));
-  w.off_x16 = at;       at = sr_align256(at + (ctx->fp16_stage ? sizeof(uint16_t) * (size_t)w.max_slots * SR_PAGE_ROWS *
-                                                                     (size_t)ctx->desc.d_model : 0));
+  w.off_x16 = at;       at = sr_align256(at + (ctx->fp16_stage || ctx->w8a8 ? (ctx->w8a8 ? 1 : 2) * (size_t)w.max_slots * SR_PAGE_ROWS *
+                                                                                     (size_t)ctx->desc.d_model : 0));
+  w.off_sx = at;        at = sr_align256(at + (ctx->w8a8 ? sizeof(float) * (size_t)w.max_slots * SR_PAGE_ROWS *
+                                                               (size_t)(ctx->desc.d_model / 128) : 0));
   at = (at + 1023) & ~size_t(1023);
   w.lane_bytes = at - lane0;
   w.lanes = lanes < 1 ? 1 : lanes;
@@ -196,6 +201,8 @@ struct SrFused {
   const __nv_bfloat16* hist;  // conv state the requests continue from, [request][C][w-1] (current layer), or null = zero
   const char* in_ssm_layer;   // recurrent states the requests continue from (current layer; slot stride below), or null
   int64_t in_ssm_slot_stride;
+  const uint8_t* x8; // W8A8 only: the layer's activation codes in slot order [slot][64][d_model], else null
+  const float* sx;   // W8A8 only: their scales [slot][d_model / 128][64]
   const __half* x16; // fp16 staging only: the layer's anchors in slot order [slot][64][d_model], else null
   const __half* w16; // fp16 staging only: dequantised k | v weight rows, then the 2 H_v gate rows, [.][d_model]
   __half* kv16;      // [slot][ncb * 128][64] = SiLU(conv(Z)) in fp16.  Rows 0..2 of a slot whose conv
@@ -244,6 +251,12 @@ cudaError_t sr_launch_anchor_write(const sr_anchor_pool& pool, const int32_t* po
 cudaError_t sr_launch_stage_weights_fp16(const sr_ctx* ctx, const sr_layer_weights& w, __half* w16, cudaStream_t stream);
 cudaError_t sr_launch_stage_anchors_fp16(const sr_ctx* ctx, const SrSched& s, const SrPoolView& pool, int32_t pool_layer,
                                          __half* x16, cudaStream_t stream);
+// W8A8: the activation quantiser (codes and scales in slot order) and, for tests, its output re-packed by request
+cudaError_t sr_launch_quant_anchors_e4m3(const sr_ctx* ctx, const SrSched& s, const SrPoolView& pool, int32_t pool_layer,
+                                         uint8_t* x8, float* sx, cudaStream_t stream);
+cudaError_t sr_launch_pack_quantised(const sr_ctx* ctx, const SrSched& s, int32_t max_pages, const uint8_t* x8,
+                                     const float* sx, void* out_codes, float* out_scales, int64_t capacity_rows,
+                                     cudaStream_t stream);
 
 // The projection with channels on the MMA's M axis and tokens on its N axis, so that each epilogue
 // thread owns one channel and walks its tokens in order: the causal conv and SiLU are applied in

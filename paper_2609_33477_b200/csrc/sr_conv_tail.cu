@@ -122,10 +122,14 @@ sr_conv_tail_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_mo
 constexpr int QT = 64;            // tile rows, tile channels and k chunk
 constexpr int QLD = QT + 8;       // shared-memory pitch (bf16)
 
-template <bool FP8>
+//   A8 (with FP8): the rows are the quantiser's activation codes instead of the bf16 anchors (W8A8): decoded to
+//                bf16 like the weight codes, and a 128-deep partial sum is scaled by weight scale x the row's
+//                activation scale of that K group.
+template <bool FP8, bool A8>
 __global__ void __launch_bounds__(128)
 sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_model, int32_t conv_ch,
                          const void* __restrict__ w_rows, const float* __restrict__ w_scale,
+                         const uint8_t* __restrict__ x8, const float* __restrict__ sx,
                          const __nv_bfloat16* __restrict__ hist, char* __restrict__ out_layer, int64_t slot_stride) {
   __shared__ __align__(16) __half Xs[2][QT * QLD];
   __shared__ __align__(16) __half Ws[2][QT * QLD];
@@ -138,45 +142,71 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
   for (int q = 0; q < 4; ++q) {
     const int m = (tid >> 3) + 16 * q;
     const int gr = r0 + m, i = gr / (SR_CONV_W - 1), j = gr % (SR_CONV_W - 1);
-    const char* src = pool.base + (int64_t)pool_layer * pool.layer_stride;       // stand-in row, masked later
+    // stand-in row (masked later): the pool's first row, or the first row of the first slot's codes
+    const char* src = A8 ? (const char*)x8 : pool.base + (int64_t)pool_layer * pool.layer_stride;
     if (i < s.n_requests && s.req_out[i] >= 0) {
       const int t = s.req_rows[i] - (SR_CONV_W - 1) + j;
       if (t >= 0) {
         const int slot = s.req_slot0[i] + t / SR_PAGE_ROWS;
-        if (sr_check_slot(s, slot) && sr_check_page(s, s.slot_page[slot]))
+        if (A8) {
+          if (sr_check_slot(s, slot)) src = (const char*)x8 + ((int64_t)slot * SR_PAGE_ROWS + t % SR_PAGE_ROWS) * d_model;
+        } else if (sr_check_slot(s, slot) && sr_check_page(s, s.slot_page[slot])) {
           src = pool.base + (int64_t)s.slot_page[slot] * pool.page_stride + (int64_t)pool_layer * pool.layer_stride +
                 (int64_t)(t % SR_PAGE_ROWS) * pool.row_stride;
+        }
       }
     }
-    xrow[q] = src + seg * 16;
+    xrow[q] = src + seg * (A8 ? 8 : 16);
     // bf16: 16 bytes = 8 weights per thread and row; e4m3: 8 bytes = 8 codes
     wrow[q] = (const char*)w_rows + ((int64_t)(c0 + m) * d_model + seg * 8) * (FP8 ? 1 : 2);
   }
-  uint2 wcode[4];                  // FP8: the next chunk's codes, in registers until their buffer is free
+  uint2 wcode[4], xcode[4];        // FP8 / A8: the next chunk's codes, in registers until their buffer is free
   auto fetch_codes = [&](int kc) {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) wcode[q] = __ldg((const uint2*)(wrow[q] + (int64_t)kc * QT));
+    for (int q = 0; q < 4; ++q) {
+      wcode[q] = __ldg((const uint2*)(wrow[q] + (int64_t)kc * QT));
+      if (A8) xcode[q] = __ldg((const uint2*)(xrow[q] + (int64_t)kc * QT));
+    }
+  };
+  auto decode_to = [&](__half* tile, int m, const uint2& codes) {
+    const uint8_t* e = (const uint8_t*)&codes;
+    __align__(16) __nv_bfloat16 o[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) o[k] = __float2bfloat16_rn(e4m3_to_float(e[k]));     // exact: 4 significant bits
+    *(uint4*)(tile + m * QLD + seg * 8) = *(const uint4*)o;
   };
   auto store_codes = [&](int b) {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int m = (tid >> 3) + 16 * q;
-      const uint8_t* e = (const uint8_t*)&wcode[q];
-      __align__(16) __nv_bfloat16 o[8];
-#pragma unroll
-      for (int k = 0; k < 8; ++k) o[k] = __float2bfloat16_rn(e4m3_to_float(e[k]));   // exact: 4 significant bits
-      *(uint4*)(Ws[b] + m * QLD + seg * 8) = *(const uint4*)o;
+      decode_to(Ws[b], m, wcode[q]);
+      if (A8) decode_to(Xs[b], m, xcode[q]);
     }
   };
   auto load = [&](int kc, int b) {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int m = (tid >> 3) + 16 * q;
-      cp_async16(Xs[b] + m * QLD + seg * 8, xrow[q] + (int64_t)kc * QT * 2);
+      if (!A8) cp_async16(Xs[b] + m * QLD + seg * 8, xrow[q] + (int64_t)kc * QT * 2);
       if (!FP8) cp_async16(Ws[b] + m * QLD + seg * 8, wrow[q] + (int64_t)kc * QT * 2);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
+  // A8: the activation scales of this thread's two accumulator rows, one float per K group (stride 64 floats)
+  const float* sxrow[2] = {sx, sx};
+  if (A8) {
+#pragma unroll
+    for (int hr = 0; hr < 2; ++hr) {
+      const int gr = r0 + warp * 16 + g8 + 8 * hr, i = gr / (SR_CONV_W - 1), j = gr % (SR_CONV_W - 1);
+      if (i < s.n_requests && s.req_out[i] >= 0) {
+        const int t = s.req_rows[i] - (SR_CONV_W - 1) + j;
+        if (t >= 0) {
+          const int slot = s.req_slot0[i] + t / SR_PAGE_ROWS;
+          if (slot >= 0 && slot < s.max_slots) sxrow[hr] = sx + (int64_t)slot * (d_model / 128) * SR_PAGE_ROWS + t % SR_PAGE_ROWS;
+        }
+      }
+    }
+  }
   float acc[8][4], total[8][4];
 #pragma unroll
   for (int n = 0; n < 8; ++n)
@@ -211,10 +241,12 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
     __syncthreads();
     if (FP8 && (kc & 1)) {         // a 128-deep k group is complete: it shares one block scale
       const float sc = __ldg(scale_row + (kc >> 1));
+      const float s0 = A8 ? sc * __ldg(sxrow[0] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
+      const float s1 = A8 ? sc * __ldg(sxrow[1] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
 #pragma unroll
       for (int n = 0; n < 8; ++n)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) { total[n][c] = fmaf(sc, acc[n][c], total[n][c]); acc[n][c] = 0.f; }
+        for (int c = 0; c < 4; ++c) { total[n][c] = fmaf(c < 2 ? s0 : s1, acc[n][c], total[n][c]); acc[n][c] = 0.f; }
     }
   }
 #pragma unroll
@@ -293,6 +325,7 @@ constexpr int GEMM_MIN_REQUESTS = 4;
 
 static bool conv_tail_gemm_fits(const sr_ctx* ctx, int n_requests) {
   const bool fp8 = ctx->desc.weight_format == SR_W_E4M3_BLOCK128;
+  if (ctx->w8a8) return true;        // quantised activations: the batched kernel is the only form (checked at sr_create)
   return (fp8 ? ctx->conv_ch : ctx->n_k) % QT == 0 && ctx->desc.d_model % (fp8 ? 128 : QT) == 0 &&
          n_requests >= GEMM_MIN_REQUESTS && !(ctx->debug_flags & SR_DEBUG_DOT_CONV_STATE);
 }
@@ -313,8 +346,14 @@ cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoo
     // every channel from codes and scales in fp32: the conv state never sees a rounded weight
     if (conv_tail_gemm_fits(ctx, s.n_requests)) {
       dim3 g((unsigned)(ctx->conv_ch / QT), (unsigned)((tail_rows + QT - 1) / QT));
-      sr_conv_tail_gemm_kernel<true><<<g, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
-                                                            w.w_qkv_scale, hist, out_conv_layer, slot_stride);
+      if (ctx->w8a8)
+        sr_conv_tail_gemm_kernel<true, true><<<g, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
+                                                                    w.w_qkv_scale, fused.x8, fused.sx, hist, out_conv_layer,
+                                                                    slot_stride);
+      else
+        sr_conv_tail_gemm_kernel<true, false><<<g, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
+                                                                     w.w_qkv_scale, nullptr, nullptr, hist, out_conv_layer,
+                                                                     slot_stride);
       return cudaGetLastError();
     }
     dim3 grid((unsigned)((ctx->conv_ch + 7) / 8), (unsigned)s.n_requests);
@@ -328,8 +367,8 @@ cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoo
   const int n_q = ctx->n_k;
   if (conv_tail_gemm_fits(ctx, s.n_requests)) {
     dim3 gq((unsigned)(n_q / QT), (unsigned)((tail_rows + QT - 1) / QT));
-    sr_conv_tail_gemm_kernel<false><<<gq, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
-                                                             nullptr, hist, out_conv_layer, slot_stride);
+    sr_conv_tail_gemm_kernel<false, false><<<gq, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
+                                                                    nullptr, nullptr, nullptr, hist, out_conv_layer, slot_stride);
     dim3 gkv((unsigned)((n_kv + 255) / 256), (unsigned)s.n_requests);
     sr_conv_tail_kv_kernel<<<gkv, 256, 0, stream>>>(s, n_q, ctx->conv_ch, zraw, n_kv, hist, out_conv_layer, slot_stride);
     return cudaGetLastError();

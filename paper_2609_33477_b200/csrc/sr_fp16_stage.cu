@@ -92,7 +92,81 @@ sr_stage_anchors_fp16_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int
   for (; i < n_vec; i += 256) convert(i, __ldcs(src(i)));
 }
 
+// W8A8: the activation quantiser.  Every row of a page slot is cut into groups of 128 consecutive channels; per
+// (row, group): s = max(amax, 1e-10) / 448 and code = e4m3(x / s), fp32 with IEEE division, round to nearest even,
+// saturating (no NaN codes).  Codes go to x8[slot][row][d] (the projection's fp8 operand, page-slot order), scales
+// to sx[slot][group][row] (one 64-float run per (slot, group), what an epilogue thread walks along its tokens).
+// Rows past the request's end get code 0 and scale 0: they contribute nothing whatever the pool holds there.
+// Half a warp per (row, group): 16 lanes x 8 values.
+__global__ void __launch_bounds__(256)
+sr_quant_anchors_e4m3_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_model, uint8_t* __restrict__ x8,
+                             float* __restrict__ sx) {
+  const int slot = blockIdx.x;
+  if (slot >= (((int)s.status[1] + 3) & ~3)) return;     // the padding slots of the last projection tile are written too
+  const int vr = s.slot_rows[slot];
+  if (vr > 0 && !sr_check_page(s, s.slot_page[slot])) return;
+  const char* page = pool.base + (int64_t)s.slot_page[slot] * pool.page_stride + (int64_t)pool_layer * pool.layer_stride;
+  const int groups = d_model / 128;
+  const int half = threadIdx.x >> 4, l16 = threadIdx.x & 15;          // 16 half-warps per CTA
+  for (int item = half; item < SR_PAGE_ROWS * groups; item += 16) {
+    const int r = item / groups, g = item % groups;
+    uint2 out = make_uint2(0u, 0u);
+    float sc = 0.f;
+    if (r < vr) {
+      const uint4 v = __ldcs((const uint4*)(page + (int64_t)r * pool.row_stride + (int64_t)g * 256 + l16 * 16));
+      const __nv_bfloat16* e = (const __nv_bfloat16*)&v;
+      float x[8], amax = 0.f;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { x[q] = __bfloat162float(e[q]); amax = fmaxf(amax, fabsf(x[q])); }
+#pragma unroll
+      for (int off = 8; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+      sc = __fdiv_rn(fmaxf(amax, 1e-10f), 448.f);
+      uint8_t c[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) c[q] = (uint8_t)__nv_cvt_float_to_fp8(__fdiv_rn(x[q], sc), __NV_SATFINITE, __NV_E4M3);
+      out = *(const uint2*)c;
+    }
+    *(uint2*)(x8 + ((int64_t)slot * SR_PAGE_ROWS + r) * d_model + g * 128 + l16 * 8) = out;
+    if (l16 == 0) sx[((int64_t)slot * groups + g) * SR_PAGE_ROWS + r] = sc;
+  }
+}
+
+// test and diagnostic: the quantiser's output re-packed by request (rows in order, no page padding)
+__global__ void __launch_bounds__(256)
+sr_pack_quantised_kernel(SrSched s, int32_t d_model, const uint8_t* __restrict__ x8, const float* __restrict__ sx,
+                         uint8_t* __restrict__ out_codes, float* __restrict__ out_scales, int64_t capacity_rows) {
+  const int i = blockIdx.y, p = blockIdx.x;
+  const int R = s.req_rows[i];
+  if (p * SR_PAGE_ROWS >= R) return;
+  const int slot = s.req_slot0[i] + p, rows = s.slot_rows[slot], groups = d_model / 128;
+  const int64_t row0 = (int64_t)s.req_row0[i] + (int64_t)p * SR_PAGE_ROWS;
+  for (int idx = threadIdx.x; idx < rows * (d_model / 16); idx += blockDim.x) {
+    const int r = idx / (d_model / 16), c16 = idx % (d_model / 16);
+    if (row0 + r < capacity_rows)
+      *(uint4*)(out_codes + (row0 + r) * d_model + c16 * 16) = *(const uint4*)(x8 + ((int64_t)slot * SR_PAGE_ROWS + r) * d_model + c16 * 16);
+  }
+  for (int idx = threadIdx.x; idx < rows * groups; idx += blockDim.x) {
+    const int r = idx / groups, g = idx % groups;
+    if (row0 + r < capacity_rows) out_scales[(row0 + r) * groups + g] = sx[((int64_t)slot * groups + g) * SR_PAGE_ROWS + r];
+  }
+}
+
 }  // namespace
+
+cudaError_t sr_launch_quant_anchors_e4m3(const sr_ctx* ctx, const SrSched& s, const SrPoolView& pool, int32_t pool_layer,
+                                         uint8_t* x8, float* sx, cudaStream_t stream) {
+  sr_quant_anchors_e4m3_kernel<<<(unsigned)s.max_slots, 256, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, x8, sx);
+  return cudaGetLastError();
+}
+
+cudaError_t sr_launch_pack_quantised(const sr_ctx* ctx, const SrSched& s, int32_t max_pages, const uint8_t* x8,
+                                     const float* sx, void* out_codes, float* out_scales, int64_t capacity_rows,
+                                     cudaStream_t stream) {
+  dim3 grid((unsigned)max_pages, (unsigned)s.n_requests);
+  sr_pack_quantised_kernel<<<grid, 256, 0, stream>>>(s, ctx->desc.d_model, x8, sx, (uint8_t*)out_codes, out_scales,
+                                                     capacity_rows);
+  return cudaGetLastError();
+}
 
 cudaError_t sr_launch_stage_weights_fp16(const sr_ctx* ctx, const sr_layer_weights& w, __half* w16, cudaStream_t stream) {
   const int d = ctx->desc.d_model;

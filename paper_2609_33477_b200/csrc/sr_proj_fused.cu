@@ -16,10 +16,12 @@
 //
 // Structure as in the plain projection: persistent, one CTA per SM, warp 0 TMA producer (one 128-channel
 // weight box and four anchor-page boxes per 64-wide k block, 4-stage ring), warp 1 tcgen05.mma issuer with
-// a double-buffered accumulator in tensor memory, epilogue warps behind.  SCALED handles e4m3 weights with
+// a double-buffered accumulator in tensor memory, epilogue warps behind.  MODE_SCALED handles e4m3 weights with
 // 128 x 128 block scales: 128-deep K groups are accumulated separately and added as scale x partial sum in
 // fp32 registers by eight epilogue warps (one scale per K group per tile, since a tile is one 128-channel
-// block).  All waits are bounded.
+// block).  MODE_W8A8 does the same on 8-bit operands: the weight codes as the caller stores them and the
+// activation codes the quantiser wrote, one 128-byte row per stage, tcgen05 kind::f8f6f4; the scale of a partial
+// sum is then weight block scale x activation scale of the token and K group.  All waits are bounded.
 #include "sr_umma.cuh"
 
 namespace {
@@ -49,6 +51,8 @@ struct FusedParams {
   int32_t act_identity;
   const float* w_scale;  // SCALED
   int32_t scale_ld;      // SCALED: d / 128
+  const float* sx;       // W8A8: activation scales [slot][d / 128][64]
+  int32_t gate_only;     // pair form: only the gate tile (the W8A8 path runs the bf16 gate rows on their own)
   const __nv_bfloat16* conv_w;
   __half* kv16;
   float* zraw;
@@ -136,8 +140,10 @@ __device__ __forceinline__ void load_history(const FusedParams& p, bool gate, in
   }
 }
 
-template <bool SCALED>
-__global__ void __launch_bounds__(SCALED ? NUM_THREADS_SCALED : NUM_THREADS, 1)
+constexpr int MODE_PLAIN = 0, MODE_SCALED = 1, MODE_W8A8 = 2;
+
+template <int MODE>
+__global__ void __launch_bounds__(MODE != MODE_PLAIN ? NUM_THREADS_SCALED : NUM_THREADS, 1)
 sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                      const __grid_constant__ CUtensorMap map_g, const FusedParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -149,10 +155,11 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   uint32_t* tmem_slot = (uint32_t*)(tempty_bar + 2);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
+  constexpr bool SCALED = MODE != MODE_PLAIN, A8 = MODE == MODE_W8A8;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_slots = (int)p.s.status[1];
   const int t_tiles = (n_slots + SLOTS - 1) / SLOTS;
-  const int c_tiles = p.n_ct + 1;
+  const int c_tiles = A8 ? p.n_ct : p.n_ct + 1;          // 8-bit operands: the bf16 gate rows go through their own launch
   const long long total_tiles = (long long)t_tiles * c_tiles;
 
   if (threadIdx.x == 0) {
@@ -196,18 +203,19 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         tile_coords(tile, ct, tt);
         int page[SLOTS];
 #pragma unroll
-        for (int q = 0; q < SLOTS; ++q) page[q] = p.fp16_stage ? SLOTS * tt + q : p.s.slot_page[SLOTS * tt + q];
+        for (int q = 0; q < SLOTS; ++q) page[q] = (p.fp16_stage || A8) ? SLOTS * tt + q : p.s.slot_page[SLOTS * tt + q];
         const bool gate = ct == p.n_ct;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
           uint8_t* a_dst = smem + stage * STAGE_BYTES;
           uint8_t* b_dst = a_dst + A_BYTES;
           mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
-          if (gate) tma_load_2d(a_dst, &map_g, &full_bar[stage], kb * BK, 0);
-          else tma_load_2d(a_dst, &map_w, &full_bar[stage], kb * BK, p.w_row0 + ct * BM);
+          const int kx = kb * (A8 ? 2 * BK : BK);         // a stage is 128 bytes of K: 64 bf16 values or 128 codes
+          if (gate) tma_load_2d(a_dst, &map_g, &full_bar[stage], kx, 0);
+          else tma_load_2d(a_dst, &map_w, &full_bar[stage], kx, p.w_row0 + ct * BM);
 #pragma unroll
           for (int q = 0; q < SLOTS; ++q)
-            tma_load_4d(b_dst + q * (B_BYTES / SLOTS), &map_x, &full_bar[stage], kb * BK, 0, p.pool_layer, page[q]);
+            tma_load_4d(b_dst + q * (B_BYTES / SLOTS), &map_x, &full_bar[stage], kx, 0, p.pool_layer, page[q]);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -219,10 +227,10 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      const uint32_t idesc = umma_idesc(BM, BN, p.fp16_stage != 0);
+      const uint32_t idesc = A8 ? umma_idesc_e4m3(BM, BN) : umma_idesc(BM, BN, p.fp16_stage != 0);
       for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        // SCALED: one accumulator buffer per 128-deep K group (2 stages); otherwise one per tile
-        const int blocks_per_acc = SCALED ? 2 : p.k_blocks;
+        // SCALED: one accumulator buffer per 128-deep K group (2 stages of bf16, 1 stage of bytes); otherwise one per tile
+        const int blocks_per_acc = A8 ? 1 : (SCALED ? 2 : p.k_blocks);
         for (int kb0 = 0; ok && kb0 < p.k_blocks; kb0 += blocks_per_acc) {
           if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -234,9 +242,10 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const uint64_t a_desc = umma_smem_desc(a_addr);
             const uint64_t b_desc = umma_smem_desc(a_addr + A_BYTES);
 #pragma unroll
-            for (int k = 0; k < BK / 16; ++k)
-              umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                        (kb != kb0 || k != 0) ? 1u : 0u);
+            for (int k = 0; k < BK / 16; ++k) {          // 32 bytes of K per instruction: 16 bf16 or 32 e4m3 values
+              if (A8) umma_e4m3(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb != kb0 || k != 0) ? 1u : 0u);
+              else umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb != kb0 || k != 0) ? 1u : 0u);
+            }
             umma_commit(&empty_bar[stage]);
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
           }
@@ -273,7 +282,9 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         float sum[128];
 #pragma unroll
         for (int i = 0; i < 128; ++i) sum[i] = 0.f;
-        const int k_groups = p.k_blocks / 2;
+        const int k_groups = A8 ? p.k_blocks : p.k_blocks / 2;
+        // W8A8: the activation scales of this warp's 128 tokens for K group kg: two runs of 64 floats (one per slot)
+        const float* sx_base = A8 ? p.sx + (long long)(SLOTS * tt + 2 * half) * k_groups * SR_PAGE_ROWS : nullptr;
         for (int kg = 0; kg < k_groups; ++kg) {
           if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag, p.s.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -283,8 +294,22 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
           for (int c = 0; c < 4; ++c) {
             float v[32];
             tmem_ld32(taddr + (uint32_t)(c * 32), v);
+            if (A8) {
+              // tokens 32 c .. 32 c + 31 of this warp's half: slot c / 2, rows 32 (c % 2) ..; the same address in
+              // every lane (a broadcast load)
+              const float4* sxp = (const float4*)(sx_base + ((long long)(c >> 1) * k_groups + kg) * SR_PAGE_ROWS + (c & 1) * 32);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) sum[c * 32 + i] = fmaf(sc, v[i], sum[c * 32 + i]);
+              for (int q = 0; q < 8; ++q) {
+                const float4 a = __ldg(sxp + q);
+                sum[c * 32 + 4 * q] = fmaf(sc * a.x, v[4 * q], sum[c * 32 + 4 * q]);
+                sum[c * 32 + 4 * q + 1] = fmaf(sc * a.y, v[4 * q + 1], sum[c * 32 + 4 * q + 1]);
+                sum[c * 32 + 4 * q + 2] = fmaf(sc * a.z, v[4 * q + 2], sum[c * 32 + 4 * q + 2]);
+                sum[c * 32 + 4 * q + 3] = fmaf(sc * a.w, v[4 * q + 3], sum[c * 32 + 4 * q + 3]);
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) sum[c * 32 + i] = fmaf(sc, v[i], sum[c * 32 + i]);
+            }
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
           __syncwarp();
@@ -360,7 +385,7 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   const int t_tiles = (n_slots + SLOTS - 1) / SLOTS;
   const int n_pt = (p.n_ct + 1) / 2;              // 256-channel tiles of k | v (the last may be half empty); tile
                                                   // index n_pt is the gate tile
-  const int c_tiles = n_pt + 1;
+  const int c_tiles = p.gate_only ? 1 : n_pt + 1;
   const long long total_tiles = (long long)t_tiles * c_tiles;
 
   if (threadIdx.x == 0) {
@@ -380,6 +405,7 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   const uint32_t tmem_base = *tmem_slot;
 
   auto tile_coords = [&](long long tile, int& pt, int& tt) {
+    if (p.gate_only) { pt = n_pt; tt = (int)tile; return; }
     const long long per_group = (long long)p.group_t * c_tiles;
     const int g = (int)(tile / per_group);
     int r = (int)(tile % per_group);
@@ -515,12 +541,14 @@ bool sr_proj_fused_exact_fp8_supported(const sr_ctx* ctx) {
 cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_anchor_pool& pool, int32_t pool_layer,
                                  const sr_layer_weights& w, const void* decoded, const SrFused& fused, int sm_count,
                                  cudaStream_t stream) {
-  // block-scaled weights: either the fp16 staging copies feed the plain kernels, or (`scaled`) bare codes with fp32
-  // promotion of the partial sums
+  // block-scaled weights: the fp16 staging copies feed the plain kernels (`stage`), or bare codes with fp32 promotion
+  // of the partial sums (`scaled`), or 8-bit operands on both sides (`a8`: quantised activations)
   const bool stage = ctx->fp16_stage;
-  const bool scaled = ctx->desc.weight_format == SR_W_E4M3_BLOCK128 && !stage;
+  const bool a8 = ctx->w8a8;
+  const bool scaled = ctx->desc.weight_format == SR_W_E4M3_BLOCK128 && !stage && !a8;
   if (scaled && !decoded) return cudaErrorInvalidValue;
   if (stage && (!fused.x16 || !fused.w16)) return cudaErrorInvalidValue;
+  if (a8 && (!fused.x8 || !fused.sx)) return cudaErrorInvalidValue;
   const int d = ctx->desc.d_model;
   const int n_kv = ctx->n_k + ctx->n_v;
   CUtensorMap map_x, map_w, map_g;
@@ -540,7 +568,7 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
     if (!encode_pool_map(&map_x, pool, d, BK)) return cudaErrorInvalidValue;
     if (scaled) {
       if (!encode_2d(&map_w, decoded, (uint64_t)d, (uint64_t)n_kv, (uint64_t)d * 2, BK, BM)) return cudaErrorInvalidValue;
-    } else {
+    } else if (!a8) {
       if (!encode_2d(&map_w, w.w_qkv, (uint64_t)d, (uint64_t)ctx->conv_ch, (uint64_t)d * 2, BK, BM)) return cudaErrorInvalidValue;
     }
     if (!encode_2d(&map_g, w.w_ab, (uint64_t)d, (uint64_t)ctx->n_gate, (uint64_t)d * 2, BK, BM)) return cudaErrorInvalidValue;
@@ -560,49 +588,77 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   p.ncb = fused.ncb;
   p.n_kv = n_kv;
   p.act_identity = ctx->desc.conv_activation == SR_CONV_IDENTITY;
-  p.w_scale = scaled ? w.w_qkv_scale : nullptr;
+  p.w_scale = (scaled || a8) ? w.w_qkv_scale : nullptr;
   p.scale_ld = d / 128;
+  p.sx = nullptr;
+  p.gate_only = 0;
   p.conv_w = (const __nv_bfloat16*)w.conv_w;
   p.kv16 = fused.kv16;
   p.zraw = fused.zraw;
   p.gates = fused.gates;
+  p.group_c = 1;
+  p.group_t = 1 << 30;
 
   cudaError_t once = sr_once_per_device(SR_ONCE_PROJ_FUSED, [] {
-    cudaError_t e = cudaFuncSetAttribute(sr_proj_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(sr_proj_fused_kernel<MODE_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(sr_proj_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+      e = cudaFuncSetAttribute(sr_proj_fused_kernel<MODE_SCALED>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(sr_proj_fused_kernel<MODE_W8A8>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(sr_proj_fused2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
     return e;
   });
   if (once != cudaSuccess) return once;
-  const long long max_tiles = (long long)(s.max_slots / SLOTS) * (p.n_ct + 1);
-  int grid = (int)(max_tiles < sm_count ? max_tiles : sm_count);
-  if (grid < 1) grid = 1;
-  // CTA pairs by default; the one-CTA form serves the exact block-scaled path and (on request) the tests
-  const bool pair_form = !scaled && sm_count >= 2 && (!(ctx->debug_flags & SR_DEBUG_SINGLE_CTA_MMA) || ctx->n_gate > BM);
+  const long long t_tiles = s.max_slots / SLOTS;
+  // CTA pairs by default; the one-CTA form serves the block-scaled forms that promote partial sums and (on request) the tests
+  const bool pair_form = !scaled && !a8 && sm_count >= 2 && (!(ctx->debug_flags & SR_DEBUG_SINGLE_CTA_MMA) || ctx->n_gate > BM);
   // Tile order: the channel tiles are cut into equal blocks of about WEIGHT_BLOCK_BYTES of weights; a block
   // stays in L2 while every token tile streams past it once (channel-fastest inside a block), so weights are
   // read from HBM once and anchors once per block.  Holding anchors instead and streaming the weights past
   // them costs more: measured 17.7 ms against 15.9 ms per launch at 254 400 tokens, d = 5120.
   {
-    const long long c_tiles = pair_form ? (p.n_ct + 1) / 2 + 1 : p.n_ct + 1;
-    const long long tile_bytes = (long long)(pair_form ? 2 * BM : BM) * d * 2;
+    const long long c_tiles = pair_form ? (p.n_ct + 1) / 2 + 1 : (a8 ? p.n_ct : p.n_ct + 1);
+    const long long tile_bytes = (long long)(pair_form ? 2 * BM : BM) * d * (a8 ? 1 : 2);
     const long long blocks = (c_tiles * tile_bytes + WEIGHT_BLOCK_BYTES - 1) / WEIGHT_BLOCK_BYTES;
     p.group_c = (int32_t)((c_tiles + blocks - 1) / blocks);
-    p.group_t = 1 << 30;
   }
-  if (pair_form) {
-    once = sr_once_per_device(SR_ONCE_PROJ_FUSED2, [] {
-      return cudaFuncSetAttribute(sr_proj_fused2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
-    });
-    if (once != cudaSuccess) return once;
-    const long long pair_tiles = (long long)(s.max_slots / SLOTS) * ((p.n_ct + 1) / 2 + 1);
+  auto launch_pairs = [&](const FusedParams& pp, long long pair_tiles) {
     long long pairs = sm_count / 2;
     if (pair_tiles < pairs) pairs = pair_tiles;
     if (pairs < 1) pairs = 1;
-    sr_proj_fused2_kernel<<<(unsigned)(2 * pairs), NUM_THREADS, SMEM2_BYTES, stream>>>(map_x, map_w, map_g, p);
+    sr_proj_fused2_kernel<<<(unsigned)(2 * pairs), NUM_THREADS, SMEM2_BYTES, stream>>>(map_x, map_w, map_g, pp);
     return cudaGetLastError();
+  };
+  if (pair_form) return launch_pairs(p, t_tiles * ((p.n_ct + 1) / 2 + 1));
+  if (a8) {
+    // (1) the bf16 gate rows on the unquantised anchors: the pair kernel restricted to its gate tile
+    if (sm_count < 2) return cudaErrorNotSupported;
+    FusedParams pg = p;
+    pg.gate_only = 1;
+    pg.w_scale = nullptr;
+    map_w = map_g;                                       // not read: every tile of this launch is the gate tile
+    cudaError_t e = launch_pairs(pg, t_tiles);
+    if (e != cudaSuccess) return e;
+    // (2) k | v on 8-bit operands: weight codes as stored, activation codes in slot order
+    sr_anchor_pool staged = pool;
+    staged.base = fused.x8;
+    staged.n_pool_layers = 1;
+    staged.n_phys_pages = s.max_slots;
+    staged.row_stride_bytes = (int64_t)d;
+    staged.layer_stride_bytes = (int64_t)SR_PAGE_ROWS * d;
+    staged.page_stride_bytes = (int64_t)SR_PAGE_ROWS * d;
+    if (!encode_pool_map(&map_x, staged, d, 2 * BK, true)) return cudaErrorInvalidValue;
+    if (!encode_2d(&map_w, w.w_qkv, (uint64_t)d, (uint64_t)ctx->conv_ch, (uint64_t)d, 2 * BK, BM, true)) return cudaErrorInvalidValue;
+    p.pool_layer = 0;
+    p.k_blocks = d / (2 * BK);
+    p.sx = fused.sx;
   }
-  if (scaled) sr_proj_fused_kernel<true><<<grid, NUM_THREADS_SCALED, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
-  else sr_proj_fused_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
+  const long long max_tiles = t_tiles * (a8 ? p.n_ct : p.n_ct + 1);
+  int grid = (int)(max_tiles < sm_count ? max_tiles : sm_count);
+  if (grid < 1) grid = 1;
+  if (a8) sr_proj_fused_kernel<MODE_W8A8><<<grid, NUM_THREADS_SCALED, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
+  else if (scaled) sr_proj_fused_kernel<MODE_SCALED><<<grid, NUM_THREADS_SCALED, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
+  else sr_proj_fused_kernel<MODE_PLAIN><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
   return cudaGetLastError();
 }

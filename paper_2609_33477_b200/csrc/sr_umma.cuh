@@ -88,6 +88,19 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a, uint64_t 
       ::"r"(tmem_d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// the same product on 8-bit operands (e4m3 x e4m3 -> fp32), K = 32 per instruction
+__device__ __forceinline__ void umma_e4m3(uint32_t tmem_d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// instruction descriptor for kind::f8f6f4 with both operands e4m3 (format code 0), D fp32, K-major, M x N
+__host__ __device__ constexpr uint32_t umma_idesc_e4m3(int m, int n) {
+  return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -198,14 +211,14 @@ inline EncodeTiledFn encode_fn() {
 }
 
 bool encode_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t row_stride_bytes,
-               uint32_t box_inner, uint32_t box_rows) {
+               uint32_t box_inner, uint32_t box_rows, bool bytes = false) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {inner, rows};
   cuuint64_t strides[1] = {row_stride_bytes};
   cuuint32_t box[2] = {box_inner, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(map, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -213,7 +226,7 @@ bool encode_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows
 
 // the pool as a 4-D tensor (column, row in page, pool layer, physical page); one box = one 64-row x
 // 64-column piece of a page, so the page-table lookup supplies the last coordinate of every load
-inline bool encode_pool_map(CUtensorMap* map, const sr_anchor_pool& pool, int d_model, uint32_t box_cols) {
+inline bool encode_pool_map(CUtensorMap* map, const sr_anchor_pool& pool, int d_model, uint32_t box_cols, bool bytes = false) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[4] = {(cuuint64_t)d_model, SR_PAGE_ROWS, (cuuint64_t)pool.n_pool_layers, (cuuint64_t)pool.n_phys_pages};
@@ -223,7 +236,7 @@ inline bool encode_pool_map(CUtensorMap* map, const sr_anchor_pool& pool, int d_
   if (pool.n_phys_pages == 1 && strides[2] == 0) strides[2] = strides[0] * SR_PAGE_ROWS;
   cuuint32_t box[4] = {box_cols, SR_PAGE_ROWS, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool.base), dims, strides, box, estr,
+  return fn(map, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool.base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

@@ -45,6 +45,7 @@ class WorkloadSpec:
     paging: str = "shuffled"          # "identity" | "shuffled" | "trunks"
     layer_mask: str = "all"           # "all" | "even"
     weight_format: str = "bf16"       # "bf16" | "e4m3_block128"
+    act_quant: str = "none"           # "none" | "e4m3_1x128" (W8A8: anchors quantised on the fly; e4m3 weights only)
     decay_scale: float = 0.1
     conv_width: int = 4
     recurrence: str = "gated_delta"   # "gated_delta" | "decay_only" (the two families of Section 2.1)
@@ -128,6 +129,12 @@ SPECS["hit_512"] = WorkloadSpec(name="hit_512", n_layers=24, d_model=2560, n_k_h
                                 d_v=128, n_requests=1, replay=("fixed", 512))
 SPECS["hits8_512"] = WorkloadSpec(name="hits8_512", n_layers=24, d_model=2560, n_k_heads=16, n_v_heads=32, d_k=128,
                                   d_v=128, n_requests=8, replay=("fixed", 512))
+# W8A8: the block-scaled configuration with on-the-fly e4m3 activations, and reduced cases of it
+SPECS["cfg4_w8a8"] = dataclasses.replace(SPECS["cfg4"], name="cfg4_w8a8", act_quant="e4m3_1x128")
+SPECS["cfg4_w8a8_slice"] = dataclasses.replace(SPECS["cfg4_slice"], name="cfg4_w8a8_slice", act_quant="e4m3_1x128")
+SPECS["w8a8_small"] = dataclasses.replace(SPECS["fp8_small"], name="w8a8_small", act_quant="e4m3_1x128")
+SPECS["w8a8_ragged"] = _spec("w8a8_ragged", 2, 1024, 4, 128, 5, ("list", (0, 3, 65, 200, 700)), weight_format="e4m3_block128",
+                             act_quant="e4m3_1x128", layer_mask="even")
 for _r in (1024, 2048, 4096):
     SPECS[f"cfg4_R{_r}"] = dataclasses.replace(SPECS["cfg4"], name=f"cfg4_R{_r}", replay=("fixed", _r))
 

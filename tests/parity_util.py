@@ -21,7 +21,8 @@ def oracle_request_layer(wl, request, layer, activation="silu", eps=1e-6, S0=Non
     arrays = synth.layer_arrays(wl.layers[layer])
     return orc.replay_request_layer(pool, pages, R, pl, arrays, n_k_heads=s.n_k_heads, n_v_heads=s.n_v_heads,
                                     d_k=s.d_k, d_v=s.d_v, eps=eps, activation=activation, S0=S0,
-                                    conv_state_bits=conv_state_bits, erase=s.recurrence != "decay_only")
+                                    conv_state_bits=conv_state_bits, erase=s.recurrence != "decay_only",
+                                    act_quant=getattr(s, "act_quant", "none"))
 
 
 def rel_frob_per_head(S_gpu, S_ref):

@@ -38,7 +38,8 @@ def _active(wl):
 
 @pytest.mark.parametrize("name", ["cfg0", "ragged_d64", "ragged_small", "trunks_small", "fp8_small", "cfg1_narrow",
                                   "grouped_small", "decay_none", "decay_strong", "grouped3_small", "wide_v_small",
-                                  "decay_only_small", "decay_only_d64", "geom_16_32", "geom_16_48", "geom_96_192"])
+                                  "decay_only_small", "decay_only_d64", "geom_16_32", "geom_16_48", "geom_96_192",
+                                  "w8a8_small", "w8a8_ragged"])
 def test_small_workloads_match_oracle_everywhere(name):
     wl, rep = _run(name)
     assert rep.device_status() == 0
@@ -93,6 +94,29 @@ def test_gather_is_bit_exact(name):
                 assert np.array_equal(got[at + t], want), (i, t)
             at += R
         assert not got[at:].any()            # nothing written past the packed rows
+
+
+def test_activation_quantiser_is_bit_exact():
+    """W8A8: the codes and scales the projection multiplies, against the oracle's quantiser on the same rows."""
+    from oracle import gdn_replay_oracle as orc
+    wl = synth.build_workload("w8a8_ragged", device=DEV)
+    rep = B.Replayer(wl)
+    for l in _active(wl):
+        codes, scales = rep.debug_quantise(l)
+        torch.cuda.synchronize()
+        codes, scales = codes.cpu().numpy(), scales.cpu().numpy()
+        at = 0
+        for i, R in enumerate(wl.replay_lens.cpu().tolist()):
+            if R == 0:
+                continue
+            pages = wl.page_table[i, : -(-R // 64)].cpu().tolist()
+            pl = wl.layer_to_pool[l]
+            X = orc.gather_anchor_rows(synth.fetch_pages(wl, pages, pl), pages, R, pl)
+            want_codes, want_scales = orc.quantise_e4m3_1x128(X)
+            assert np.array_equal(codes[at:at + R], want_codes), (l, i)
+            assert np.array_equal(scales[at:at + R], want_scales), (l, i)
+            at += R
+        assert not codes[at:].any() and not scales[at:].any()
 
 
 def test_masked_layers_and_other_slots_are_not_touched():
