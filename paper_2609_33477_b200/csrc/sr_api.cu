@@ -333,7 +333,8 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
     fused.ncb = (ctx->n_k + ctx->n_v + 127) / 128;
     fused.n_kv = ctx->n_k + ctx->n_v;
     fused.n_gate = ctx->n_gate;
-    fused.fix_mod = (d.weight_format == SR_W_E4M3_BLOCK128 && !ctx->fp16_stage) ? 2 : 4;
+    // page slots per run of the projection's conv epilogue (the first three rows of a run are finished by the scan)
+    fused.fix_mod = ctx->w8a8 ? 1 : ((d.weight_format == SR_W_E4M3_BLOCK128 && !ctx->fp16_stage) ? 2 : 4);
     fused.hist = nullptr;
     fused.in_ssm_layer = nullptr;
     fused.in_ssm_slot_stride = 0;

@@ -52,7 +52,7 @@ struct sr_ctx {
 // calls return cudaSuccess at once.  A failed set-up is retried by the next call.
 enum SrOnceKey {
   SR_ONCE_PROJ_FUSED = 0, SR_ONCE_PROJ_FUSED2, SR_ONCE_CHUNK_LOCAL_64, SR_ONCE_CHUNK_LOCAL_96,
-  SR_ONCE_CHUNK_LOCAL_128, SR_ONCE_CHAIN_UMMA, SR_ONCE_KEYS
+  SR_ONCE_CHUNK_LOCAL_128, SR_ONCE_CHAIN_UMMA, SR_ONCE_CONV_GEMM, SR_ONCE_KEYS
 };
 cudaError_t sr_once_per_device(int key, cudaError_t (*setup)());
 // SM count of the current device (looked up once per device)

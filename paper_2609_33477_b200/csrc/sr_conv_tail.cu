@@ -121,6 +121,12 @@ sr_conv_tail_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_mo
 //                state of block-scaled layers is as exact as the one of bf16 layers.
 constexpr int QT = 64;            // tile rows, tile channels and k chunk
 constexpr int QLD = QT + 8;       // shared-memory pitch (bf16)
+constexpr int QNS = 4;            // chunks in flight: the k loop is serial, so its speed is latency / depth
+
+template <bool FP8, bool A8>
+constexpr int conv_gemm_smem() {
+  return ((A8 ? 2 : QNS) + (FP8 ? 2 : QNS)) * QT * QLD * 2 + ((A8 ? QNS : 0) + (FP8 ? QNS : 0)) * QT * QT;
+}
 
 //   A8 (with FP8): the rows are the quantiser's activation codes instead of the bf16 anchors (W8A8): decoded to
 //                bf16 like the weight codes, and a 128-deep partial sum is scaled by weight scale x the row's
@@ -131,8 +137,15 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
                          const void* __restrict__ w_rows, const float* __restrict__ w_scale,
                          const uint8_t* __restrict__ x8, const float* __restrict__ sx,
                          const __nv_bfloat16* __restrict__ hist, char* __restrict__ out_layer, int64_t slot_stride) {
-  __shared__ __align__(16) __half Xs[2][QT * QLD];
-  __shared__ __align__(16) __half Ws[2][QT * QLD];
+  // Shared memory: a ring of QNS stages per operand.  A 16-bit operand is copied straight into its padded tile
+  // (cp.async, 16 bytes); an 8-bit operand lands as raw bytes (cp.async, 8 bytes) and the thread that fetched them
+  // decodes them into one of two bf16 tiles just before the chunk is used.
+  extern __shared__ __align__(16) uint8_t qsm[];
+  constexpr int TILE_B = QT * QLD * 2, RAW_B = QT * QT;
+  __half* Xt = (__half*)qsm;                                              // [A8 ? 2 : QNS] tiles
+  __half* Wt = (__half*)(qsm + (A8 ? 2 : QNS) * TILE_B);                  // [FP8 ? 2 : QNS] tiles
+  uint8_t* Xraw = qsm + ((A8 ? 2 : QNS) + (FP8 ? 2 : QNS)) * TILE_B;      // [QNS] raw chunks (A8)
+  uint8_t* Wraw = Xraw + (A8 ? QNS * RAW_B : 0);                          // [QNS] raw chunks (FP8)
   const int tid = threadIdx.x, warp = tid >> 5, l = tid & 31, g8 = l >> 2, t4 = l & 3;
   const int c0 = blockIdx.x * QT, r0 = blockIdx.y * QT;
   const int seg = tid & 7;
@@ -160,37 +173,28 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
     // bf16: 16 bytes = 8 weights per thread and row; e4m3: 8 bytes = 8 codes
     wrow[q] = (const char*)w_rows + ((int64_t)(c0 + m) * d_model + seg * 8) * (FP8 ? 1 : 2);
   }
-  uint2 wcode[4], xcode[4];        // FP8 / A8: the next chunk's codes, in registers until their buffer is free
-  auto fetch_codes = [&](int kc) {
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      wcode[q] = __ldg((const uint2*)(wrow[q] + (int64_t)kc * QT));
-      if (A8) xcode[q] = __ldg((const uint2*)(xrow[q] + (int64_t)kc * QT));
-    }
-  };
-  auto decode_to = [&](__half* tile, int m, const uint2& codes) {
-    const uint8_t* e = (const uint8_t*)&codes;
-    __align__(16) __nv_bfloat16 o[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) o[k] = __float2bfloat16_rn(e4m3_to_float(e[k]));     // exact: 4 significant bits
-    *(uint4*)(tile + m * QLD + seg * 8) = *(const uint4*)o;
-  };
-  auto store_codes = [&](int b) {
+  auto load = [&](int kc) {            // chunk kc -> ring stage kc % QNS
+    const int st = kc % QNS;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int m = (tid >> 3) + 16 * q;
-      decode_to(Ws[b], m, wcode[q]);
-      if (A8) decode_to(Xs[b], m, xcode[q]);
+      if (A8) cp_async8(Xraw + st * RAW_B + m * QT + seg * 8, xrow[q] + (int64_t)kc * QT);
+      else cp_async16(Xt + st * (QT * QLD) + m * QLD + seg * 8, xrow[q] + (int64_t)kc * QT * 2);
+      if (FP8) cp_async8(Wraw + st * RAW_B + m * QT + seg * 8, wrow[q] + (int64_t)kc * QT);
+      else cp_async16(Wt + st * (QT * QLD) + m * QLD + seg * 8, wrow[q] + (int64_t)kc * QT * 2);
     }
   };
-  auto load = [&](int kc, int b) {
+  auto decode_own = [&](const uint8_t* raw, __half* tile) {      // this thread's own bytes: no barrier needed before
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int m = (tid >> 3) + 16 * q;
-      if (!A8) cp_async16(Xs[b] + m * QLD + seg * 8, xrow[q] + (int64_t)kc * QT * 2);
-      if (!FP8) cp_async16(Ws[b] + m * QLD + seg * 8, wrow[q] + (int64_t)kc * QT * 2);
+      const uint2 codes = *(const uint2*)(raw + m * QT + seg * 8);
+      const uint8_t* e = (const uint8_t*)&codes;
+      __align__(16) __nv_bfloat16 o[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) o[k] = __float2bfloat16_rn(e4m3_to_float(e[k]));     // exact: 4 significant bits
+      *(uint4*)(tile + m * QLD + seg * 8) = *(const uint4*)o;
     }
-    asm volatile("cp.async.commit_group;" ::: "memory");
   };
   // A8: the activation scales of this thread's two accumulator rows, one float per K group (stride 64 floats)
   const float* sxrow[2] = {sx, sx};
@@ -214,31 +218,30 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
     for (int c = 0; c < 4; ++c) { acc[n][c] = 0.f; total[n][c] = 0.f; }
   const int nk = d_model / QT;
   const float* scale_row = FP8 ? w_scale + (int64_t)(c0 / 128) * (d_model / 128) : nullptr;
-  load(0, 0);
-  if (FP8) fetch_codes(0);
+  for (int kc = 0; kc < QNS - 1; ++kc) {       // fill the ring; one commit group per chunk, empty ones past the end
+    if (kc < nk) load(kc);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
   for (int kc = 0; kc < nk; ++kc) {
-    const int b = kc & 1;
-    if (FP8) store_codes(b);       // buffer b was last read two chunks ago; a barrier closed that chunk
-    if (kc + 1 < nk) {
-      load(kc + 1, b ^ 1);
-      if (FP8) fetch_codes(kc + 1);
-      asm volatile("cp.async.wait_group 1;" ::: "memory");
-    } else {
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
-    }
-    __syncthreads();
+    asm volatile("cp.async.wait_group %0;" ::"n"(QNS - 2) : "memory");      // this thread's part of chunk kc has landed
+    const __half* xt = A8 ? Xt + (kc & 1) * (QT * QLD) : Xt + (kc % QNS) * (QT * QLD);
+    const __half* wt = FP8 ? Wt + (kc & 1) * (QT * QLD) : Wt + (kc % QNS) * (QT * QLD);
+    if (A8) decode_own(Xraw + (kc % QNS) * RAW_B, (__half*)xt);
+    if (FP8) decode_own(Wraw + (kc % QNS) * RAW_B, (__half*)wt);
+    __syncthreads();                  // chunk kc is complete for everyone; everyone is done with chunk kc - 1
+    if (kc + QNS - 1 < nk) load(kc + QNS - 1);                             // into the stage chunk kc - 1 used
+    asm volatile("cp.async.commit_group;" ::: "memory");
 #pragma unroll
     for (int ks = 0; ks < QT / 16; ++ks) {
       uint32_t a[4], bf[4];
-      ldsm4(a, a_addr(Xs[b], QLD, warp * 16, ks * 16, l));
+      ldsm4(a, a_addr(xt, QLD, warp * 16, ks * 16, l));
 #pragma unroll
       for (int nb = 0; nb < 4; ++nb) {
-        ldsm4(bf, bn_addr(Ws[b], QLD, nb * 16, ks * 16, l));
+        ldsm4(bf, bn_addr(wt, QLD, nb * 16, ks * 16, l));
         mma16816_bf16(acc[2 * nb], a, bf[0], bf[1]);
         mma16816_bf16(acc[2 * nb + 1], a, bf[2], bf[3]);
       }
     }
-    __syncthreads();
     if (FP8 && (kc & 1)) {         // a 128-deep k group is complete: it shares one block scale
       const float sc = __ldg(scale_row + (kc >> 1));
       const float s0 = A8 ? sc * __ldg(sxrow[0] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
@@ -318,16 +321,13 @@ sr_hist_gather_kernel(SrSched s, const char* __restrict__ in_layer, int64_t slot
 
 // kernels one sr_launch_conv_tail call launches: bf16 weights, the batched q GEMM plus the k | v copy; block-scaled
 // weights, one GEMM over all channels; geometries the 64-wide tiles do not divide, the single dot-product kernel
-// The GEMM reads every weight once per 64 tail rows but walks d_model serially in one CTA per 64 channels; below
-// GEMM_MIN_REQUESTS requests the dot-product kernel (a warp per channel and request, thousands of short chains)
-// finishes sooner.
-constexpr int GEMM_MIN_REQUESTS = 4;
-
+// The batched kernel serves every batch size its tiles divide, so that a request's conv state has the same bits
+// whatever batch it arrives in.
 static bool conv_tail_gemm_fits(const sr_ctx* ctx, int n_requests) {
   const bool fp8 = ctx->desc.weight_format == SR_W_E4M3_BLOCK128;
   if (ctx->w8a8) return true;        // quantised activations: the batched kernel is the only form (checked at sr_create)
   return (fp8 ? ctx->conv_ch : ctx->n_k) % QT == 0 && ctx->desc.d_model % (fp8 ? 128 : QT) == 0 &&
-         n_requests >= GEMM_MIN_REQUESTS && !(ctx->debug_flags & SR_DEBUG_DOT_CONV_STATE);
+         !(ctx->debug_flags & SR_DEBUG_DOT_CONV_STATE);
 }
 
 int sr_conv_tail_launches(const sr_ctx* ctx, int n_requests) {
@@ -342,16 +342,28 @@ cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoo
   const __nv_bfloat16* hist = fused.hist;
   const int n_kv = ctx->n_k + ctx->n_v;
   const int tail_rows = s.n_requests * (SR_CONV_W - 1);
+  const cudaError_t once = sr_once_per_device(SR_ONCE_CONV_GEMM, [] {
+    cudaError_t e = cudaFuncSetAttribute(sr_conv_tail_gemm_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         conv_gemm_smem<false, false>());
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(sr_conv_tail_gemm_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               conv_gemm_smem<true, false>());
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(sr_conv_tail_gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               conv_gemm_smem<true, true>());
+    return e;
+  });
+  if (once != cudaSuccess) return once;
   if (ctx->desc.weight_format == SR_W_E4M3_BLOCK128) {
     // every channel from codes and scales in fp32: the conv state never sees a rounded weight
     if (conv_tail_gemm_fits(ctx, s.n_requests)) {
       dim3 g((unsigned)(ctx->conv_ch / QT), (unsigned)((tail_rows + QT - 1) / QT));
       if (ctx->w8a8)
-        sr_conv_tail_gemm_kernel<true, true><<<g, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
+        sr_conv_tail_gemm_kernel<true, true><<<g, 128, conv_gemm_smem<true, true>(), stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
                                                                     w.w_qkv_scale, fused.x8, fused.sx, hist, out_conv_layer,
                                                                     slot_stride);
       else
-        sr_conv_tail_gemm_kernel<true, false><<<g, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
+        sr_conv_tail_gemm_kernel<true, false><<<g, 128, conv_gemm_smem<true, false>(), stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
                                                                      w.w_qkv_scale, nullptr, nullptr, hist, out_conv_layer,
                                                                      slot_stride);
       return cudaGetLastError();
@@ -367,7 +379,7 @@ cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoo
   const int n_q = ctx->n_k;
   if (conv_tail_gemm_fits(ctx, s.n_requests)) {
     dim3 gq((unsigned)(n_q / QT), (unsigned)((tail_rows + QT - 1) / QT));
-    sr_conv_tail_gemm_kernel<false, false><<<gq, 128, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
+    sr_conv_tail_gemm_kernel<false, false><<<gq, 128, conv_gemm_smem<false, false>(), stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
                                                                     nullptr, nullptr, nullptr, hist, out_conv_layer, slot_stride);
     dim3 gkv((unsigned)((n_kv + 255) / 256), (unsigned)s.n_requests);
     sr_conv_tail_kv_kernel<<<gkv, 256, 0, stream>>>(s, n_q, ctx->conv_ch, zraw, n_kv, hist, out_conv_layer, slot_stride);

@@ -37,6 +37,9 @@ __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefe
 __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
 }
+__device__ __forceinline__ void cp_async8(void* dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
 // fragment addresses (lane l): see the m16n8k16 operand layouts
 __device__ __forceinline__ const __half* a_addr(const __half* base, int ld, int row0, int col0, int l) {       // A from [M][K]
   return base + (row0 + (l & 15)) * ld + col0 + (l >> 4) * 8;

@@ -16,12 +16,10 @@
 //
 // Structure as in the plain projection: persistent, one CTA per SM, warp 0 TMA producer (one 128-channel
 // weight box and four anchor-page boxes per 64-wide k block, 4-stage ring), warp 1 tcgen05.mma issuer with
-// a double-buffered accumulator in tensor memory, epilogue warps behind.  MODE_SCALED handles e4m3 weights with
+// a double-buffered accumulator in tensor memory, epilogue warps behind.  SCALED handles e4m3 weights with
 // 128 x 128 block scales: 128-deep K groups are accumulated separately and added as scale x partial sum in
 // fp32 registers by eight epilogue warps (one scale per K group per tile, since a tile is one 128-channel
-// block).  MODE_W8A8 does the same on 8-bit operands: the weight codes as the caller stores them and the
-// activation codes the quantiser wrote, one 128-byte row per stage, tcgen05 kind::f8f6f4; the scale of a partial
-// sum is then weight block scale x activation scale of the token and K group.  All waits are bounded.
+// block).  sr_proj_w8a8_kernel (below) runs the 8-bit form.  All waits are bounded.
 #include "sr_umma.cuh"
 
 namespace {
@@ -140,10 +138,8 @@ __device__ __forceinline__ void load_history(const FusedParams& p, bool gate, in
   }
 }
 
-constexpr int MODE_PLAIN = 0, MODE_SCALED = 1, MODE_W8A8 = 2;
-
-template <int MODE>
-__global__ void __launch_bounds__(MODE != MODE_PLAIN ? NUM_THREADS_SCALED : NUM_THREADS, 1)
+template <bool SCALED>
+__global__ void __launch_bounds__(SCALED ? NUM_THREADS_SCALED : NUM_THREADS, 1)
 sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                      const __grid_constant__ CUtensorMap map_g, const FusedParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -155,11 +151,10 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   uint32_t* tmem_slot = (uint32_t*)(tempty_bar + 2);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
-  constexpr bool SCALED = MODE != MODE_PLAIN, A8 = MODE == MODE_W8A8;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_slots = (int)p.s.status[1];
   const int t_tiles = (n_slots + SLOTS - 1) / SLOTS;
-  const int c_tiles = A8 ? p.n_ct : p.n_ct + 1;          // 8-bit operands: the bf16 gate rows go through their own launch
+  const int c_tiles = p.n_ct + 1;
   const long long total_tiles = (long long)t_tiles * c_tiles;
 
   if (threadIdx.x == 0) {
@@ -203,19 +198,18 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         tile_coords(tile, ct, tt);
         int page[SLOTS];
 #pragma unroll
-        for (int q = 0; q < SLOTS; ++q) page[q] = (p.fp16_stage || A8) ? SLOTS * tt + q : p.s.slot_page[SLOTS * tt + q];
+        for (int q = 0; q < SLOTS; ++q) page[q] = p.fp16_stage ? SLOTS * tt + q : p.s.slot_page[SLOTS * tt + q];
         const bool gate = ct == p.n_ct;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
           uint8_t* a_dst = smem + stage * STAGE_BYTES;
           uint8_t* b_dst = a_dst + A_BYTES;
           mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
-          const int kx = kb * (A8 ? 2 * BK : BK);         // a stage is 128 bytes of K: 64 bf16 values or 128 codes
-          if (gate) tma_load_2d(a_dst, &map_g, &full_bar[stage], kx, 0);
-          else tma_load_2d(a_dst, &map_w, &full_bar[stage], kx, p.w_row0 + ct * BM);
+          if (gate) tma_load_2d(a_dst, &map_g, &full_bar[stage], kb * BK, 0);
+          else tma_load_2d(a_dst, &map_w, &full_bar[stage], kb * BK, p.w_row0 + ct * BM);
 #pragma unroll
           for (int q = 0; q < SLOTS; ++q)
-            tma_load_4d(b_dst + q * (B_BYTES / SLOTS), &map_x, &full_bar[stage], kx, 0, p.pool_layer, page[q]);
+            tma_load_4d(b_dst + q * (B_BYTES / SLOTS), &map_x, &full_bar[stage], kb * BK, 0, p.pool_layer, page[q]);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -227,10 +221,10 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      const uint32_t idesc = A8 ? umma_idesc_e4m3(BM, BN) : umma_idesc(BM, BN, p.fp16_stage != 0);
+      const uint32_t idesc = umma_idesc(BM, BN, p.fp16_stage != 0);
       for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        // SCALED: one accumulator buffer per 128-deep K group (2 stages of bf16, 1 stage of bytes); otherwise one per tile
-        const int blocks_per_acc = A8 ? 1 : (SCALED ? 2 : p.k_blocks);
+        // SCALED: one accumulator buffer per 128-deep K group (2 stages); otherwise one per tile
+        const int blocks_per_acc = SCALED ? 2 : p.k_blocks;
         for (int kb0 = 0; ok && kb0 < p.k_blocks; kb0 += blocks_per_acc) {
           if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -242,10 +236,9 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const uint64_t a_desc = umma_smem_desc(a_addr);
             const uint64_t b_desc = umma_smem_desc(a_addr + A_BYTES);
 #pragma unroll
-            for (int k = 0; k < BK / 16; ++k) {          // 32 bytes of K per instruction: 16 bf16 or 32 e4m3 values
-              if (A8) umma_e4m3(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb != kb0 || k != 0) ? 1u : 0u);
-              else umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb != kb0 || k != 0) ? 1u : 0u);
-            }
+            for (int k = 0; k < BK / 16; ++k)
+              umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                        (kb != kb0 || k != 0) ? 1u : 0u);
             umma_commit(&empty_bar[stage]);
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
           }
@@ -282,9 +275,7 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         float sum[128];
 #pragma unroll
         for (int i = 0; i < 128; ++i) sum[i] = 0.f;
-        const int k_groups = A8 ? p.k_blocks : p.k_blocks / 2;
-        // W8A8: the activation scales of this warp's 128 tokens for K group kg: two runs of 64 floats (one per slot)
-        const float* sx_base = A8 ? p.sx + (long long)(SLOTS * tt + 2 * half) * k_groups * SR_PAGE_ROWS : nullptr;
+        const int k_groups = p.k_blocks / 2;
         for (int kg = 0; kg < k_groups; ++kg) {
           if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag, p.s.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -294,22 +285,8 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
           for (int c = 0; c < 4; ++c) {
             float v[32];
             tmem_ld32(taddr + (uint32_t)(c * 32), v);
-            if (A8) {
-              // tokens 32 c .. 32 c + 31 of this warp's half: slot c / 2, rows 32 (c % 2) ..; the same address in
-              // every lane (a broadcast load)
-              const float4* sxp = (const float4*)(sx_base + ((long long)(c >> 1) * k_groups + kg) * SR_PAGE_ROWS + (c & 1) * 32);
 #pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                const float4 a = __ldg(sxp + q);
-                sum[c * 32 + 4 * q] = fmaf(sc * a.x, v[4 * q], sum[c * 32 + 4 * q]);
-                sum[c * 32 + 4 * q + 1] = fmaf(sc * a.y, v[4 * q + 1], sum[c * 32 + 4 * q + 1]);
-                sum[c * 32 + 4 * q + 2] = fmaf(sc * a.z, v[4 * q + 2], sum[c * 32 + 4 * q + 2]);
-                sum[c * 32 + 4 * q + 3] = fmaf(sc * a.w, v[4 * q + 3], sum[c * 32 + 4 * q + 3]);
-              }
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) sum[c * 32 + i] = fmaf(sc, v[i], sum[c * 32 + i]);
-            }
+            for (int i = 0; i < 32; ++i) sum[c * 32 + i] = fmaf(sc, v[i], sum[c * 32 + i]);
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
           __syncwarp();
@@ -340,6 +317,215 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         __syncwarp();
         if (lane == 0) mbar_arrive(&tempty_bar[acc]);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// W8A8: e4m3 weight codes (as the caller stores them) x e4m3 activation codes (written by the quantiser, page-slot
+// order), tcgen05 kind::f8f6f4, one 128-byte row of K per stage.  Both operands carry block scales that are plain
+// fp32 numbers, not the hardware's power-of-two block format, so every 128-deep K group has to enter the result as
+//     total[channel][token] += w_scale[channel block][group] * x_scale[token][group] * partial[channel][token]
+// outside the tensor core.  Keeping `total` in registers (128 values per epilogue thread) spills; here it lives in
+// tensor memory next to the partial sums: columns 0..127 and 128..255 hold the partial sums of the tile's two token
+// halves (each half its own MMA of N = 128 and its own full / empty barriers, so the halves pipeline against each
+// other), columns 256..511 hold the totals.  An epilogue warp owns 32 lanes x 64 columns of each half: it loads a
+// chunk of partial sums and the matching chunk of totals, does the multiply-add with the scale products shared
+// through shared memory, and stores the totals back.  After the last group the same warp runs the conv + SiLU
+// epilogue on its two page slots (slots hw and hw + 2 of the tile's four: their conv history lies with another
+// warp, so every slot's first three rows are finished later, like the first rows of a tile in the 16-bit kernels).
+constexpr int W8_BK = 128;                       // bytes (= codes) of K per stage
+constexpr int W8_NH = BN / 2;                    // tokens per half tile
+constexpr int W8_SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + 2 * 2 * BN * 4;
+
+__global__ void __launch_bounds__(NUM_THREADS_SCALED, 1)
+sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const FusedParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* full_bar = (uint64_t*)(smem + STAGES * STAGE_BYTES);
+  uint64_t* empty_bar = full_bar + STAGES;
+  uint64_t* pfull_bar = empty_bar + STAGES;      // [2] partial sums of a token half complete
+  uint64_t* pempty_bar = pfull_bar + 2;          // [2] ... drained by the eight epilogue warps
+  uint64_t* sx_full = pempty_bar + 2;            // [2] activation scales of a K group landed
+  uint32_t* tmem_slot = (uint32_t*)(sx_full + 2);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+  float* sxs = (float*)(smem + STAGES * STAGE_BYTES + 256);      // [2][BN] activation scales of a K group
+  float* comb = sxs + 2 * BN;                                    // [2][BN] weight scale x activation scale
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_slots = (int)p.s.status[1];
+  const int t_tiles = (n_slots + SLOTS - 1) / SLOTS;
+  const int c_tiles = p.n_ct;                    // the bf16 gate rows go through their own launch
+  const long long total_tiles = (long long)t_tiles * c_tiles;
+  const int k_groups = p.k_blocks;               // one stage = one 128-deep group
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&pfull_bar[i], 1); mbar_init(&pempty_bar[i], 8); mbar_init(&sx_full[i], 1); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  auto tile_coords = [&](long long tile, int& ct, int& tt) {     // same walk as the 16-bit kernels
+    const long long per_group = (long long)p.group_t * c_tiles;
+    const int g = (int)(tile / per_group);
+    int r = (int)(tile % per_group);
+    const int gt = min(p.group_t, t_tiles - g * p.group_t);
+    const int per_block = gt * p.group_c;
+    const int cb = r / per_block;
+    r -= cb * per_block;
+    const int gc = min(p.group_c, c_tiles - cb * p.group_c);
+    ct = cb * p.group_c + r % gc;
+    tt = g * p.group_t + r / gc;
+  };
+
+  if (warp == 0) {
+    if (lane == 0) {                             // TMA producer
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        int ct, tt;
+        tile_coords(tile, ct, tt);
+        for (int kb = 0; kb < k_groups; ++kb) {
+          if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
+          uint8_t* a_dst = smem + stage * STAGE_BYTES;
+          uint8_t* b_dst = a_dst + A_BYTES;
+          mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
+          tma_load_2d(a_dst, &map_w, &full_bar[stage], kb * W8_BK, p.w_row0 + ct * BM);
+#pragma unroll
+          for (int q = 0; q < SLOTS; ++q)
+            tma_load_4d(b_dst + q * (B_BYTES / SLOTS), &map_x, &full_bar[stage], kb * W8_BK, 0, 0, SLOTS * tt + q);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {                             // MMA issue
+      int stage = 0;
+      uint32_t phase = 0, gcount = 0;
+      bool ok = true;
+      const uint32_t idesc = umma_idesc_e4m3(BM, W8_NH);
+      for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        int ct, tt;
+        tile_coords(tile, ct, tt);
+        for (int kg = 0; ok && kg < k_groups; ++kg, ++gcount) {
+          const uint32_t b = gcount & 1u, par = (gcount >> 1) & 1u;
+          for (int h = 0; h < 2; ++h) {
+            // the epilogue has drained this half's partial sums of the previous group
+            if (!mbar_wait(&pempty_bar[h], ((gcount & 1u) ^ 1u), abort_flag, p.s.status)) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (h == 0) {
+              // ... which also means the group before that is finished everywhere: its scale buffer is free.  Fetch this
+              // group's activation scales (one 64-float run per page slot) while the MMAs run.
+              mbar_expect_tx(&sx_full[b], BN * 4);
+#pragma unroll
+              for (int q = 0; q < SLOTS; ++q)
+                bulk_load(sxs + b * BN + q * SR_PAGE_ROWS, p.sx + ((long long)(SLOTS * tt + q) * k_groups + kg) * SR_PAGE_ROWS,
+                          SR_PAGE_ROWS * 4, &sx_full[b]);
+              if (!mbar_wait(&full_bar[stage], phase, abort_flag, p.s.status)) { ok = false; break; }
+              asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            }
+            const uint32_t a_addr = smem_u32(smem + stage * STAGE_BYTES);
+            const uint64_t a_desc = umma_smem_desc(a_addr);
+            const uint64_t b_desc = umma_smem_desc(a_addr + A_BYTES + h * (B_BYTES / 2));
+#pragma unroll
+            for (int k = 0; k < W8_BK / 32; ++k)
+              umma_e4m3(tmem_base + (uint32_t)(h * W8_NH), a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, k != 0 ? 1u : 0u);
+            umma_commit(&pfull_bar[h]);
+          }
+          (void)par;
+          if (!ok) break;
+          umma_commit(&empty_bar[stage]);        // the stage is free once both halves' products have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // epilogue: tensor-memory lanes 32 * (warp % 4) .., columns hw * 64 .. of each token half
+    const int quarter = warp & 3, hw = (warp - 2) >> 2;
+    const int ch_local = quarter * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const int e = (warp - 2) * 32 + lane;        // 0..255: this thread's entry of the scale products
+    uint32_t gcount = 0;
+    bool ok = true;
+    for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      int ct, tt;
+      tile_coords(tile, ct, tt);
+      const int ch = ct * BM + ch_local;
+      const float* scale_row = p.w_scale + (long long)((p.n_q + ct * BM) / 128) * p.scale_ld;
+      for (int kg = 0; kg < k_groups; ++kg, ++gcount) {
+        const uint32_t b = gcount & 1u, par_sx = (gcount >> 1) & 1u, par_p = gcount & 1u;
+        // weight scale x activation scale for the tile's 256 tokens: one product per epilogue thread
+        if (ok) ok = mbar_wait(&sx_full[b], par_sx, abort_flag, p.s.status);
+        comb[b * BN + e] = ok ? __ldg(scale_row + kg) * sxs[b * BN + e] : 0.f;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (ok) ok = mbar_wait(&pfull_bar[h], par_p, abort_flag, p.s.status);
+          if (ok) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t col = (uint32_t)(h * W8_NH + hw * 64);
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              float v[32], t[32];
+              tmem_ld32_issue(tmem_base + lane_off + col + (uint32_t)(c * 32), v);
+              if (kg > 0) tmem_ld32_issue(tmem_base + lane_off + (uint32_t)BN + col + (uint32_t)(c * 32), t);
+              tmem_wait_ld();
+              const float4* cb = (const float4*)(comb + b * BN + col + c * 32);      // same address in every lane
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                const float4 a = cb[q];
+                t[4 * q] = kg > 0 ? fmaf(a.x, v[4 * q], t[4 * q]) : a.x * v[4 * q];
+                t[4 * q + 1] = kg > 0 ? fmaf(a.y, v[4 * q + 1], t[4 * q + 1]) : a.y * v[4 * q + 1];
+                t[4 * q + 2] = kg > 0 ? fmaf(a.z, v[4 * q + 2], t[4 * q + 2]) : a.z * v[4 * q + 2];
+                t[4 * q + 3] = kg > 0 ? fmaf(a.w, v[4 * q + 3], t[4 * q + 3]) : a.w * v[4 * q + 3];
+              }
+              tmem_st32(tmem_base + lane_off + (uint32_t)BN + col + (uint32_t)(c * 32), t);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+          }
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&pempty_bar[h]);      // also after a failed wait: nobody is left waiting on this warp
+        }
+      }
+      // One decision for all eight warps (they meet at the named barrier once per group, so none may leave alone):
+      // a wait that gave up anywhere in the CTA has raised the flag.
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (*abort_flag) break;
+      // the tile's totals are complete: conv + SiLU on this warp's two page slots
+      float cw[4] = {0.f, 0.f, 0.f, 0.f};
+      if (ch < p.n_kv) {
+        const uint2 wv = *(const uint2*)(p.conv_w + (long long)(p.n_q + ch) * SR_CONV_W);
+        const __nv_bfloat16* w4 = (const __nv_bfloat16*)&wv;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) cw[q] = __bfloat162float(w4[q]);
+      }
+#pragma unroll 1
+      for (int sl = hw; sl < SLOTS; sl += 2) {
+        const int slot = SLOTS * tt + sl;
+        float v[64], z1, z2, z3;
+        tmem_ld32(tmem_base + lane_off + (uint32_t)(BN + sl * 64), v);
+        tmem_ld32(tmem_base + lane_off + (uint32_t)(BN + sl * 64 + 32), v + 32);
+        load_history(p, false, p.s.slot_first[slot], ch, z1, z2, z3);
+        emit_slot(p, false, ch, ch_local, ct, slot, true, p.s.slot_rows[slot], v, cw, z1, z2, z3);
       }
     }
   }
@@ -600,11 +786,11 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   p.group_t = 1 << 30;
 
   cudaError_t once = sr_once_per_device(SR_ONCE_PROJ_FUSED, [] {
-    cudaError_t e = cudaFuncSetAttribute(sr_proj_fused_kernel<MODE_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(sr_proj_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(sr_proj_fused_kernel<MODE_SCALED>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+      e = cudaFuncSetAttribute(sr_proj_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(sr_proj_fused_kernel<MODE_W8A8>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+      e = cudaFuncSetAttribute(sr_proj_w8a8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, W8_SMEM_BYTES);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(sr_proj_fused2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
     return e;
@@ -657,8 +843,8 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   const long long max_tiles = t_tiles * (a8 ? p.n_ct : p.n_ct + 1);
   int grid = (int)(max_tiles < sm_count ? max_tiles : sm_count);
   if (grid < 1) grid = 1;
-  if (a8) sr_proj_fused_kernel<MODE_W8A8><<<grid, NUM_THREADS_SCALED, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
-  else if (scaled) sr_proj_fused_kernel<MODE_SCALED><<<grid, NUM_THREADS_SCALED, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
-  else sr_proj_fused_kernel<MODE_PLAIN><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
+  if (a8) sr_proj_w8a8_kernel<<<grid, NUM_THREADS_SCALED, W8_SMEM_BYTES, stream>>>(map_x, map_w, p);
+  else if (scaled) sr_proj_fused_kernel<true><<<grid, NUM_THREADS_SCALED, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
+  else sr_proj_fused_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
   return cudaGetLastError();
 }
