@@ -34,7 +34,9 @@ the functions below are pinned by tests, the *choices* are "parity unpinned"):
     projections; value head h uses key head h // (H_v / H_k);
   * the conv state lists, per channel, the last w-1 projection rows oldest first.
 
-The sidecar's write side (anchor_write: destination-table indexed stores, Section 5.1) is restated too.
+The sidecar's write side (anchor_write: destination-table indexed stores, Section 5.1) is restated too, and so is
+group-propagated replay (Section 4.1: one anchor per group of consecutive linear-attention layers; block_forward,
+gated_delta_outputs, group_replay) -- the latter as this build's reading of a block the paper does not spell out.
 
 Pins (tests/test_oracle_pins.py): exact rational arithmetic on tiny projections, the
 unrolled sum of Eq. 5 by explicit matrix products, closed forms for one-hot and
@@ -44,7 +46,9 @@ recurrence, of the convolution with its history, and of a whole layer replayed i
 pieces against one pass), the contraction bound of the replay error, library convolution /
 activation routines, all 256 e4m3 codes, the e4m3 activation quantiser (codes and scales bit for bit
 against a library cast, every representable value as a fixed point, ties and saturation, the half-step
-error bound), the state sizes printed in the paper's Appendix A table, and a write / gather round trip.
+error bound), the state sizes printed in the paper's Appendix A table, a write / gather round trip; for group
+replay: per-token outputs against the unrolled state of Eq. 5, the causal-linear-attention limit as one masked
+matrix product, the block against a library composition, and the layer-to-layer feeding of a group.
 """
 
 from __future__ import annotations
@@ -337,6 +341,93 @@ def replay_request_layer(pool, pages, n_rows, pool_layer, arrays: dict, *, n_k_h
     return replay_layer(X, w_qkv, w_ab, conv_w, c, delta, n_k_heads=n_k_heads, n_v_heads=n_v_heads,
                         d_k=d_k, d_v=d_v, eps=eps, activation=activation, S0=S0, conv_state_bits=conv_state_bits,
                         erase=erase, act_quant=act_quant)
+
+
+# ---------------------------------------------------------------------------------------
+# Group-propagated replay (Section 4.1, "Layer-wise Sparse Anchors"): one anchor per GROUP of consecutive
+# linear-attention layers.  Only the hidden state entering the group's first layer is stored; replay rebuilds the
+# first layer's state from it and, to feed the next layer of the group, also has to produce that layer's OUTPUT
+# for every replayed row -- the per-token half of the layer that single-layer replay never computes.
+#
+# The paper describes the scheme, not the block, so the block below is this build's reading (a pre-norm residual
+# block around a gated-delta mixer, the shape hybrid models of this family use; every choice "parity unpinned"):
+#
+#   x_t  = RMSNorm(r_t; norm_w)                               layer input, from the residual stream r_t
+#   q, k, v, alpha, beta from x_t as in replay_layer; q is L2-normalised like k and scaled by d_k^-1/2
+#   o_t[h] = S_t[h]^T q_t[kh]                                  read-out of the state AFTER the update at t
+#   g_t  = x_t W_z^T                                           output gate, H_v d_v wide
+#   y_t  = RMSNorm_per_head(o_t; o_norm_w) * SiLU(g_t)
+#   r'_t = bf16(r_t + y_t W_o^T)                               residual add, stored in bf16
+#   r''_t = bf16(r'_t + (SiLU(n W_gate^T) * (n W_up^T)) W_down^T),  n = RMSNorm(r'_t; mlp_norm_w)    (optional MLP)
+#
+# The group's anchors are rows of the residual stream entering its first layer.
+
+def rms_norm(x, w, eps: float = 1e-6) -> np.ndarray:
+    x = np.asarray(x, dtype=np.float64)
+    return x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps) * np.asarray(w, dtype=np.float64)
+
+
+def gated_delta_outputs(q, k_hat, v, alpha, beta, S0=None, erase: bool = True):
+    """The recurrence of gated_delta_recurrence with the per-token read-out o_t = S_t^T q_t (the state after the
+    update at t).  q [R, H_k, d_k]; returns (O [R, H_v, d_v], S [H_v, d_k, d_v])."""
+    q = np.asarray(q, dtype=np.float64)
+    k_hat = np.asarray(k_hat, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    R, H_k, d_k = k_hat.shape
+    _, H_v, d_v = v.shape
+    group = H_v // H_k
+    S = np.zeros((H_v, d_k, d_v)) if S0 is None else np.array(S0, dtype=np.float64)
+    O = np.zeros((R, H_v, d_v))
+    for t in range(R):
+        k_t = np.repeat(k_hat[t], group, axis=0)
+        q_t = np.repeat(q[t], group, axis=0)
+        S = alpha[t][:, None, None] * S
+        r = np.einsum("hkv,hk->hv", S, k_t) if erase else 0.0
+        S = S + beta[t][:, None, None] * k_t[:, :, None] * (v[t] - r)[:, None, :]
+        O[t] = np.einsum("hkv,hk->hv", S, q_t)
+    return O, S
+
+
+def block_forward(r_rows, layer: dict, *, n_k_heads, n_v_heads, d_k, d_v, eps: float = 1e-6, norm_eps: float = 1e-6,
+                  erase: bool = True):
+    """One block of a group on the residual-stream rows r [R, d] (fp64 values of bf16 storage).
+
+    `layer`: fp64 arrays norm_w [d], w_qkv [C, d], w_ab [2 H_v, d], conv_w [C, w], decay_scale, dt_bias [H_v],
+    w_z [H_v d_v, d], o_norm_w [d_v], w_o [d, H_v d_v] and optionally mlp_norm_w [d], w_gate, w_up [f, d],
+    w_down [d, f].  Returns (next residual rows as bf16 bits [R, d], S fp32 [H_v, d_k, d_v], conv state bits)."""
+    r_rows = np.asarray(r_rows, dtype=np.float64)
+    R = r_rows.shape[0]
+    x = rms_norm(r_rows, layer["norm_w"], norm_eps)
+    Z, G = in_projection(x, layer["w_qkv"], layer["w_ab"])
+    width = np.asarray(layer["conv_w"]).shape[1]
+    tail = conv_tail_bits(Z, width)
+    Y = causal_conv_silu(Z, layer["conv_w"])
+    q, k, v = split_qkv(Y, n_k_heads, n_v_heads, d_k, d_v)
+    alpha, beta = gates(G, layer["decay_scale"], layer["dt_bias"])
+    O, S = gated_delta_outputs(l2_normalise(q, eps) * d_k ** -0.5, l2_normalise(k, eps), v, alpha, beta, erase=erase)
+    gate = x @ np.asarray(layer["w_z"], dtype=np.float64).T
+    y = (rms_norm(O, layer["o_norm_w"], norm_eps).reshape(R, n_v_heads * d_v)) * (gate / (1.0 + np.exp(-gate)))
+    r1 = bf16_bits_to_f64(f64_to_bf16_bits(r_rows + y @ np.asarray(layer["w_o"], dtype=np.float64).T))
+    if "w_gate" in layer:
+        n = rms_norm(r1, layer["mlp_norm_w"], norm_eps)
+        a = n @ np.asarray(layer["w_gate"], dtype=np.float64).T
+        hidden = (a / (1.0 + np.exp(-a))) * (n @ np.asarray(layer["w_up"], dtype=np.float64).T)
+        r1 = bf16_bits_to_f64(f64_to_bf16_bits(r1 + hidden @ np.asarray(layer["w_down"], dtype=np.float64).T))
+    return f64_to_bf16_bits(r1), S.astype(np.float32), tail
+
+
+def group_replay(anchor_rows, layers, **geometry):
+    """States of every layer of one group from the group-entry anchors alone (Section 4.1): layer j is replayed on
+    the rows that layers 0..j-1 of the group produced.  anchor_rows [R, d] fp64 (residual stream entering the
+    group); returns [(S fp32, conv state bits)] per layer.  The last layer's output is never formed."""
+    r = np.asarray(anchor_rows, dtype=np.float64)
+    out = []
+    for j, layer in enumerate(layers):
+        bits, S, tail = block_forward(r, layer, **geometry)
+        out.append((S, tail))
+        if j + 1 < len(layers):
+            r = bf16_bits_to_f64(bits)
+    return out
 
 
 # ---------------------------------------------------------------------------------------

@@ -624,6 +624,125 @@ def test_replay_request_layer_reads_pages_through_the_table():
     assert np.all(S0 == 0) and np.all(tail0 == 0) and tail0.shape == (C, 3)
 
 
+# ----------------------------------------------------------------- group-propagated replay (Section 4.1)
+
+def _group_layer(r, d, Hk, Hv, dk, dv, mlp=0):
+    C = 2 * Hk * dk + Hv * dv
+    L = dict(norm_w=r.uniform(0.5, 1.5, d), w_qkv=r.standard_normal((C, d)) / math.sqrt(d),
+             w_ab=r.standard_normal((2 * Hv, d)) / math.sqrt(d), conv_w=r.standard_normal((C, 4)) / 2,
+             decay_scale=np.full(Hv, 0.1), dt_bias=np.zeros(Hv), w_z=r.standard_normal((Hv * dv, d)) / math.sqrt(d),
+             o_norm_w=r.uniform(0.5, 1.5, dv), w_o=r.standard_normal((d, Hv * dv)) / math.sqrt(Hv * dv))
+    if mlp:
+        L.update(mlp_norm_w=r.uniform(0.5, 1.5, d), w_gate=r.standard_normal((mlp, d)) / math.sqrt(d),
+                 w_up=r.standard_normal((mlp, d)) / math.sqrt(d), w_down=r.standard_normal((d, mlp)) / math.sqrt(mlp))
+    return L
+
+
+def test_rms_norm_matches_the_library():
+    r = _rng(70)
+    x, w = r.standard_normal((5, 3, 16)), r.uniform(0.5, 2, 16)
+    lib = torch.nn.functional.rms_norm(torch.from_numpy(x), (16,), torch.from_numpy(w), eps=1e-6).numpy()
+    assert np.allclose(orc.rms_norm(x, w), lib, rtol=1e-13, atol=1e-15)
+
+
+def test_per_token_outputs_are_the_read_out_of_the_unrolled_state():
+    """o_t = S_t^T q_t with S_t from Eq. 5 by explicit transition products; and the final state is the recurrence's."""
+    r = _rng(71)
+    R, Hk, Hv, dk, dv = 9, 2, 4, 5, 3
+    q = r.standard_normal((R, Hk, dk))
+    k = _unit_rows(r.standard_normal((R, Hk, dk)))
+    v = r.standard_normal((R, Hv, dv))
+    alpha, beta = r.uniform(0.5, 1, (R, Hv)), r.uniform(0, 1, (R, Hv))
+    O, S = orc.gated_delta_outputs(q, k, v, alpha, beta)
+    assert np.allclose(S, orc.gated_delta_recurrence(k, v, alpha, beta), rtol=0, atol=1e-15)
+    for h in range(Hv):
+        kh = h // 2
+        for t in range(R):
+            St = np.zeros((dk, dv))
+            for i in range(t + 1):
+                B = beta[i, h] * np.outer(k[i, kh], v[i, h])
+                for j in range(i + 1, t + 1):
+                    B = alpha[j, h] * (np.eye(dk) - beta[j, h] * np.outer(k[j, kh], k[j, kh])) @ B
+                St += B
+            assert np.allclose(O[t, h], St.T @ q[t, kh], rtol=1e-11, atol=1e-13)
+
+
+def test_outputs_without_erase_and_decay_are_causal_linear_attention():
+    """erase off, alpha = 1: o_t = sum_{s <= t} beta_s (k_s . q_t) v_s, one masked matrix product."""
+    r = _rng(72)
+    R, dk, dv = 12, 6, 4
+    q, k, v = r.standard_normal((R, 1, dk)), r.standard_normal((R, 1, dk)), r.standard_normal((R, 1, dv))
+    beta = r.uniform(0, 1, (R, 1))
+    O, _ = orc.gated_delta_outputs(q, k, v, np.ones((R, 1)), beta, erase=False)
+    want = np.tril(q[:, 0] @ k[:, 0].T) @ (beta * v[:, 0])
+    assert np.allclose(O[:, 0], want, rtol=1e-12, atol=1e-13)
+
+
+def test_block_against_a_library_composition_and_single_row_closed_form():
+    r = _rng(73)
+    R, d, Hk, Hv, dk, dv = 13, 32, 2, 4, 4, 6
+    geo = dict(n_k_heads=Hk, n_v_heads=Hv, d_k=dk, d_v=dv)
+    L = _group_layer(r, d, Hk, Hv, dk, dv, mlp=24)
+    rows = torch.from_numpy(r.standard_normal((R, d))).to(torch.bfloat16).double()
+    bits, S, tail = orc.block_forward(rows.numpy(), L, **geo)
+    T = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
+    F = torch.nn.functional
+    x = F.rms_norm(rows, (d,), T(L["norm_w"]), eps=1e-6)
+    Z = F.linear(x, T(L["w_qkv"]))
+    C = Z.shape[1]
+    Y = F.silu(F.conv1d(F.pad(Z.T[None], (3, 0)), T(L["conv_w"])[:, None, :], groups=C))[0].T
+    nq = Hk * dk
+    q, k, v = Y[:, :nq].reshape(R, Hk, dk), Y[:, nq:2 * nq].reshape(R, Hk, dk), Y[:, 2 * nq:].reshape(R, Hv, dv)
+    q = q / torch.sqrt((q * q).sum(-1, keepdim=True) + 1e-6) * dk ** -0.5
+    k = k / torch.sqrt((k * k).sum(-1, keepdim=True) + 1e-6)
+    G = F.linear(x, T(L["w_ab"]))
+    alpha, beta = torch.exp(-0.1 * F.softplus(G[:, :Hv])), torch.sigmoid(G[:, Hv:])
+    St = torch.zeros(Hv, dk, dv, dtype=torch.float64)
+    O = torch.zeros(R, Hv, dv, dtype=torch.float64)
+    for t in range(R):
+        for h in range(Hv):
+            kk = k[t, h // 2]
+            St[h] = alpha[t, h] * (torch.eye(dk, dtype=torch.float64) - beta[t, h] * torch.outer(kk, kk)) @ St[h] \
+                + beta[t, h] * torch.outer(kk, v[t, h])
+            O[t, h] = St[h].T @ q[t, h // 2]
+    y = (F.rms_norm(O, (dv,), T(L["o_norm_w"]), eps=1e-6).reshape(R, Hv * dv)) * F.silu(F.linear(x, T(L["w_z"])))
+    r1 = (rows + F.linear(y, T(L["w_o"]))).to(torch.bfloat16).double()
+    n = F.rms_norm(r1, (d,), T(L["mlp_norm_w"]), eps=1e-6)
+    r2 = (r1 + F.linear(F.silu(F.linear(n, T(L["w_gate"]))) * F.linear(n, T(L["w_up"])), T(L["w_down"]))).to(torch.bfloat16)
+    got = orc.bf16_bits_to_f64(bits)
+    dist = np.abs(got - r2.double().numpy())
+    assert (dist == 0).mean() > 0.99 and np.all(dist <= np.abs(got) * 2.0 ** -7 + 1e-30)   # bf16 ties may flip a bit
+    assert np.allclose(S, St.numpy().astype(np.float32), rtol=1e-6, atol=1e-9)
+    assert np.array_equal(tail, _bf16_bits(Z[-3:].T.float()))
+    # the state and conv state are those of single-layer replay on the normed rows
+    S1, tail1 = orc.replay_layer(x.numpy(), L["w_qkv"], L["w_ab"], L["conv_w"], L["decay_scale"], L["dt_bias"], **geo)
+    assert np.array_equal(S, S1) and np.array_equal(tail, tail1)
+
+
+def test_group_replay_feeds_each_layer_with_the_previous_block_output():
+    r = _rng(74)
+    R, d, Hk, Hv, dk, dv = 10, 32, 2, 2, 4, 4
+    geo = dict(n_k_heads=Hk, n_v_heads=Hv, d_k=dk, d_v=dv)
+    layers = [_group_layer(r, d, Hk, Hv, dk, dv, mlp=(16 if j == 1 else 0)) for j in range(3)]
+    anchors = torch.from_numpy(r.standard_normal((R, d))).to(torch.bfloat16).double().numpy()
+    res = orc.group_replay(anchors, layers, **geo)
+    assert len(res) == 3
+    rows = anchors
+    for j, L in enumerate(layers):
+        bits, S, tail = orc.block_forward(rows, L, **geo)
+        assert np.array_equal(res[j][0], S) and np.array_equal(res[j][1], tail)
+        rows = orc.bf16_bits_to_f64(bits)
+    # layers of a group are coupled only through the rows: changing layer 0's output projection changes the states of
+    # layers 1 and 2 but not layer 0's
+    layers2 = [dict(layers[0], w_o=layers[0]["w_o"] * 1.5)] + layers[1:]
+    res2 = orc.group_replay(anchors, layers2, **geo)
+    assert np.array_equal(res2[0][0], res[0][0])
+    assert not np.allclose(res2[1][0], res[1][0]) and not np.allclose(res2[2][0], res[2][0])
+    # a single-layer group is single-layer replay of the normed anchors
+    one = orc.group_replay(anchors, layers[:1], **geo)
+    assert np.array_equal(one[0][0], res[0][0])
+
+
 # ----------------------------------------------------------------- sizes the paper prints
 
 def test_state_extents_reproduce_appendix_a_table():
