@@ -163,7 +163,8 @@ def oracle_one(wl, req, layer, rows):
     arrays = synth.layer_arrays(wl.layers[layer])
     t0 = time.perf_counter()
     S, _ = orc.replay_request_layer(pool, pages, rows, pl, arrays, n_k_heads=s.n_k_heads, n_v_heads=s.n_v_heads,
-                                    d_k=s.d_k, d_v=s.d_v)
+                                    d_k=s.d_k, d_v=s.d_v, erase=s.recurrence != "decay_only",
+                                    act_quant=getattr(s, "act_quant", "none"))
     dt = time.perf_counter() - t0
     assert np.all(np.isfinite(S))
     return dt

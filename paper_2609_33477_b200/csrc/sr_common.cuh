@@ -16,7 +16,7 @@
 #define SR_PAGE_ROWS 64
 #define SR_CONV_W 4
 #define SR_MAX_LANES 4                       // layers in flight at once on small batches
-#define SR_LANES_BUDGET_BYTES (512ull << 20) // ... as long as their hand-over buffers together stay below this
+#define SR_LANES_BUDGET_BYTES (1024ull << 20) // ... as long as their hand-over buffers together stay below this
 
 struct sr_ctx {
   sr_model_desc desc;

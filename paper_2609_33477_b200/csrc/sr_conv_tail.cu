@@ -196,26 +196,36 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
       *(uint4*)(tile + m * QLD + seg * 8) = *(const uint4*)o;
     }
   };
-  // A8: the activation scales of this thread's two accumulator rows, one float per K group (stride 64 floats)
-  const float* sxrow[2] = {sx, sx};
-  if (A8) {
+  // Work split: warp w owns channels 16 w .. 16 w + 15 of the tile for every 16-row block that holds a tail row (the
+  // tail rows of a tile are its first n_rb blocks), so one weight fragment serves four row blocks and the products of
+  // a step do not wait on one another.  A thread's accumulator rows: 16 rb + g8 and 16 rb + g8 + 8.
+  const int rows_here = min(QT, s.n_requests * (SR_CONV_W - 1) - r0);
+  const int n_rb = (rows_here + 15) / 16;
+  // A8: the activation scales of those rows, one float per K group (stride 64 floats)
+  const float* sxrow[4][2];
+#pragma unroll
+  for (int rb = 0; rb < 4; ++rb)
 #pragma unroll
     for (int hr = 0; hr < 2; ++hr) {
-      const int gr = r0 + warp * 16 + g8 + 8 * hr, i = gr / (SR_CONV_W - 1), j = gr % (SR_CONV_W - 1);
-      if (i < s.n_requests && s.req_out[i] >= 0) {
-        const int t = s.req_rows[i] - (SR_CONV_W - 1) + j;
-        if (t >= 0) {
-          const int slot = s.req_slot0[i] + t / SR_PAGE_ROWS;
-          if (slot >= 0 && slot < s.max_slots) sxrow[hr] = sx + (int64_t)slot * (d_model / 128) * SR_PAGE_ROWS + t % SR_PAGE_ROWS;
+      sxrow[rb][hr] = sx;
+      if (A8) {
+        const int gr = r0 + rb * 16 + g8 + 8 * hr, i = gr / (SR_CONV_W - 1), j = gr % (SR_CONV_W - 1);
+        if (i < s.n_requests && s.req_out[i] >= 0) {
+          const int t = s.req_rows[i] - (SR_CONV_W - 1) + j;
+          if (t >= 0) {
+            const int slot = s.req_slot0[i] + t / SR_PAGE_ROWS;
+            if (slot >= 0 && slot < s.max_slots) sxrow[rb][hr] = sx + (int64_t)slot * (d_model / 128) * SR_PAGE_ROWS + t % SR_PAGE_ROWS;
+          }
         }
       }
     }
-  }
-  float acc[8][4], total[8][4];
+  float acc[4][2][4], total[4][2][4];
 #pragma unroll
-  for (int n = 0; n < 8; ++n)
+  for (int rb = 0; rb < 4; ++rb)
 #pragma unroll
-    for (int c = 0; c < 4; ++c) { acc[n][c] = 0.f; total[n][c] = 0.f; }
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) { acc[rb][n][c] = 0.f; total[rb][n][c] = 0.f; }
   const int nk = d_model / QT;
   const float* scale_row = FP8 ? w_scale + (int64_t)(c0 / 128) * (d_model / 128) : nullptr;
   for (int kc = 0; kc < QNS - 1; ++kc) {       // fill the ring; one commit group per chunk, empty ones past the end
@@ -233,46 +243,57 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
     asm volatile("cp.async.commit_group;" ::: "memory");
 #pragma unroll
     for (int ks = 0; ks < QT / 16; ++ks) {
-      uint32_t a[4], bf[4];
-      ldsm4(a, a_addr(xt, QLD, warp * 16, ks * 16, l));
+      uint32_t bf[4];
+      ldsm4(bf, bn_addr(wt, QLD, warp * 16, ks * 16, l));
 #pragma unroll
-      for (int nb = 0; nb < 4; ++nb) {
-        ldsm4(bf, bn_addr(wt, QLD, nb * 16, ks * 16, l));
-        mma16816_bf16(acc[2 * nb], a, bf[0], bf[1]);
-        mma16816_bf16(acc[2 * nb + 1], a, bf[2], bf[3]);
+      for (int rb = 0; rb < 4; ++rb) {
+        if (rb < n_rb) {
+          uint32_t a[4];
+          ldsm4(a, a_addr(xt, QLD, rb * 16, ks * 16, l));
+          mma16816_bf16(acc[rb][0], a, bf[0], bf[1]);
+          mma16816_bf16(acc[rb][1], a, bf[2], bf[3]);
+        }
       }
     }
     if (FP8 && (kc & 1)) {         // a 128-deep k group is complete: it shares one block scale
       const float sc = __ldg(scale_row + (kc >> 1));
-      const float s0 = A8 ? sc * __ldg(sxrow[0] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
-      const float s1 = A8 ? sc * __ldg(sxrow[1] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
 #pragma unroll
-      for (int n = 0; n < 8; ++n)
+      for (int rb = 0; rb < 4; ++rb) {
+        if (rb < n_rb) {
+          const float s0 = A8 ? sc * __ldg(sxrow[rb][0] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
+          const float s1 = A8 ? sc * __ldg(sxrow[rb][1] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) { total[n][c] = fmaf(c < 2 ? s0 : s1, acc[n][c], total[n][c]); acc[n][c] = 0.f; }
+          for (int n = 0; n < 2; ++n)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) { total[rb][n][c] = fmaf(c < 2 ? s0 : s1, acc[rb][n][c], total[rb][n][c]); acc[rb][n][c] = 0.f; }
+        }
+      }
     }
   }
 #pragma unroll
-  for (int hr = 0; hr < 2; ++hr) {
-    const int gr = r0 + warp * 16 + g8 + 8 * hr, i = gr / (SR_CONV_W - 1), j = gr % (SR_CONV_W - 1);
-    if (i >= s.n_requests) continue;
-    const int out_slot = s.req_out[i];
-    if (out_slot < 0 || !sr_check_out(s, out_slot)) continue;
-    const int t = s.req_rows[i] - (SR_CONV_W - 1) + j;
-    // rows before the window: zero, or the inputs of the state this request continues (kept bit for bit)
-    const __nv_bfloat16* old = (t < 0 && hist) ? hist + (int64_t)i * conv_ch * (SR_CONV_W - 1) + (SR_CONV_W - 1 + t) : nullptr;
-    __nv_bfloat16* dst = (__nv_bfloat16*)(out_layer + (int64_t)out_slot * slot_stride) + j;
+  for (int rb = 0; rb < 4; ++rb) {
 #pragma unroll
-    for (int n = 0; n < 8; ++n) {
-      const int c = c0 + n * 8 + 2 * t4;
-      const float v0 = FP8 ? total[n][2 * hr] : acc[n][2 * hr], v1 = FP8 ? total[n][2 * hr + 1] : acc[n][2 * hr + 1];
-      __nv_bfloat16 o0 = __float2bfloat16_rn(t >= 0 ? v0 : 0.f), o1 = __float2bfloat16_rn(t >= 0 ? v1 : 0.f);
-      if (old) {
-        o0 = old[(int64_t)c * (SR_CONV_W - 1)];
-        o1 = old[(int64_t)(c + 1) * (SR_CONV_W - 1)];
+    for (int hr = 0; hr < 2; ++hr) {
+      const int gr = r0 + rb * 16 + g8 + 8 * hr, i = gr / (SR_CONV_W - 1), j = gr % (SR_CONV_W - 1);
+      if (rb >= n_rb || i >= s.n_requests) continue;
+      const int out_slot = s.req_out[i];
+      if (out_slot < 0 || !sr_check_out(s, out_slot)) continue;
+      const int t = s.req_rows[i] - (SR_CONV_W - 1) + j;
+      // rows before the window: zero, or the inputs of the state this request continues (kept bit for bit)
+      const __nv_bfloat16* old = (t < 0 && hist) ? hist + (int64_t)i * conv_ch * (SR_CONV_W - 1) + (SR_CONV_W - 1 + t) : nullptr;
+      __nv_bfloat16* dst = (__nv_bfloat16*)(out_layer + (int64_t)out_slot * slot_stride) + j;
+#pragma unroll
+      for (int n = 0; n < 2; ++n) {
+        const int c = c0 + warp * 16 + n * 8 + 2 * t4;
+        const float v0 = FP8 ? total[rb][n][2 * hr] : acc[rb][n][2 * hr], v1 = FP8 ? total[rb][n][2 * hr + 1] : acc[rb][n][2 * hr + 1];
+        __nv_bfloat16 o0 = __float2bfloat16_rn(t >= 0 ? v0 : 0.f), o1 = __float2bfloat16_rn(t >= 0 ? v1 : 0.f);
+        if (old) {
+          o0 = old[(int64_t)c * (SR_CONV_W - 1)];
+          o1 = old[(int64_t)(c + 1) * (SR_CONV_W - 1)];
+        }
+        dst[(int64_t)c * (SR_CONV_W - 1)] = o0;
+        dst[(int64_t)(c + 1) * (SR_CONV_W - 1)] = o1;
       }
-      dst[(int64_t)c * (SR_CONV_W - 1)] = o0;
-      dst[(int64_t)(c + 1) * (SR_CONV_W - 1)] = o1;
     }
   }
 }
