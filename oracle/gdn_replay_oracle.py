@@ -397,7 +397,8 @@ def block_forward(r_rows, layer: dict, *, n_k_heads, n_v_heads, d_k, d_v, eps: f
     w_down [d, f].  Returns (next residual rows as bf16 bits [R, d], S fp32 [H_v, d_k, d_v], conv state bits)."""
     r_rows = np.asarray(r_rows, dtype=np.float64)
     R = r_rows.shape[0]
-    x = rms_norm(r_rows, layer["norm_w"], norm_eps)
+    # the layer input stands where a stored anchor stands in single-layer replay: a bf16 hidden state
+    x = bf16_bits_to_f64(f64_to_bf16_bits(rms_norm(r_rows, layer["norm_w"], norm_eps)))
     Z, G = in_projection(x, layer["w_qkv"], layer["w_ab"])
     width = np.asarray(layer["conv_w"]).shape[1]
     tail = conv_tail_bits(Z, width)
@@ -409,25 +410,27 @@ def block_forward(r_rows, layer: dict, *, n_k_heads, n_v_heads, d_k, d_v, eps: f
     y = (rms_norm(O, layer["o_norm_w"], norm_eps).reshape(R, n_v_heads * d_v)) * (gate / (1.0 + np.exp(-gate)))
     r1 = bf16_bits_to_f64(f64_to_bf16_bits(r_rows + y @ np.asarray(layer["w_o"], dtype=np.float64).T))
     if "w_gate" in layer:
-        n = rms_norm(r1, layer["mlp_norm_w"], norm_eps)
+        n = bf16_bits_to_f64(f64_to_bf16_bits(rms_norm(r1, layer["mlp_norm_w"], norm_eps)))
         a = n @ np.asarray(layer["w_gate"], dtype=np.float64).T
         hidden = (a / (1.0 + np.exp(-a))) * (n @ np.asarray(layer["w_up"], dtype=np.float64).T)
         r1 = bf16_bits_to_f64(f64_to_bf16_bits(r1 + hidden @ np.asarray(layer["w_down"], dtype=np.float64).T))
     return f64_to_bf16_bits(r1), S.astype(np.float32), tail
 
 
-def group_replay(anchor_rows, layers, **geometry):
+def group_replay(anchor_rows, layers, return_rows: bool = False, **geometry):
     """States of every layer of one group from the group-entry anchors alone (Section 4.1): layer j is replayed on
     the rows that layers 0..j-1 of the group produced.  anchor_rows [R, d] fp64 (residual stream entering the
-    group); returns [(S fp32, conv state bits)] per layer.  The last layer's output is never formed."""
+    group); returns [(S fp32, conv state bits)] per layer.  The last layer's output is never formed.  With
+    return_rows also the bf16 bits of the rows handed from each layer to the next ([R, d] per hand-over)."""
     r = np.asarray(anchor_rows, dtype=np.float64)
-    out = []
+    out, handed = [], []
     for j, layer in enumerate(layers):
         bits, S, tail = block_forward(r, layer, **geometry)
         out.append((S, tail))
         if j + 1 < len(layers):
+            handed.append(bits)
             r = bf16_bits_to_f64(bits)
-    return out
+    return (out, handed) if return_rows else out
 
 
 # ---------------------------------------------------------------------------------------

@@ -687,7 +687,7 @@ def test_block_against_a_library_composition_and_single_row_closed_form():
     bits, S, tail = orc.block_forward(rows.numpy(), L, **geo)
     T = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
     F = torch.nn.functional
-    x = F.rms_norm(rows, (d,), T(L["norm_w"]), eps=1e-6)
+    x = F.rms_norm(rows, (d,), T(L["norm_w"]), eps=1e-6).to(torch.bfloat16).double()   # layer inputs are bf16, like anchors
     Z = F.linear(x, T(L["w_qkv"]))
     C = Z.shape[1]
     Y = F.silu(F.conv1d(F.pad(Z.T[None], (3, 0)), T(L["conv_w"])[:, None, :], groups=C))[0].T
@@ -707,7 +707,7 @@ def test_block_against_a_library_composition_and_single_row_closed_form():
             O[t, h] = St[h].T @ q[t, h // 2]
     y = (F.rms_norm(O, (dv,), T(L["o_norm_w"]), eps=1e-6).reshape(R, Hv * dv)) * F.silu(F.linear(x, T(L["w_z"])))
     r1 = (rows + F.linear(y, T(L["w_o"]))).to(torch.bfloat16).double()
-    n = F.rms_norm(r1, (d,), T(L["mlp_norm_w"]), eps=1e-6)
+    n = F.rms_norm(r1, (d,), T(L["mlp_norm_w"]), eps=1e-6).to(torch.bfloat16).double()
     r2 = (r1 + F.linear(F.silu(F.linear(n, T(L["w_gate"]))) * F.linear(n, T(L["w_up"])), T(L["w_down"]))).to(torch.bfloat16)
     got = orc.bf16_bits_to_f64(bits)
     dist = np.abs(got - r2.double().numpy())
