@@ -314,6 +314,58 @@ int sr_replay_states_host(sr_ctx* ctx, const void* host_pool, size_t pool_bytes,
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Group-propagated replay (Section 4.1, "Layer-wise Sparse Anchors": the hidden state is stored only at the entry
+ * of each group of consecutive linear-attention layers; replay rebuilds the states of all the group's layers from
+ * that one anchor, running the linear-attention layers of the group in sequence and never a full-attention layer).
+ *
+ * To feed layer j + 1 of a group the call has to produce layer j's OUTPUT for every replayed row, which single-layer
+ * replay never computes.  The paper does not spell the block out; this library takes a pre-norm residual block
+ * around the gated-delta mixer (the shape hybrid models of this family use), with r the residual-stream row:
+ *
+ *   x = RMSNorm(r; norm_w)                    the layer input: q, k, v, alpha, beta and both states as in sr_replay_states
+ *   q^ = q / sqrt(|q|^2 + l2_eps) / sqrt(d_k);   o[h] = S_t[h]^T q^[key head of h]     (state after the update at t)
+ *   y  = RMSNorm(o[h]; o_norm_w) * SiLU(x W_z^T)                                       (per value head)
+ *   r' = bf16(r + y W_o^T)
+ *   r''= bf16(r' + (SiLU(n W_gate^T) * (n W_up^T)) W_down^T),  n = RMSNorm(r'; mlp_norm_w)    if an MLP is given
+ *
+ * and the next layer of the group takes r'' (or r') as its residual-stream row.  RMSNorm(v; w) = v / sqrt(mean(v^2) +
+ * norm_eps) * w.  The anchors of the group are the residual-stream rows entering its FIRST layer: pool layer
+ * layer_to_pool[first_layer].
+ *
+ * One layer of a group: HOST struct holding DEVICE pointers, all bf16, K (input width) contiguous.
+ */
+typedef struct sr_block_weights {
+  const void* norm_w;      /* [d_model]                                              */
+  const void* w_z;         /* [H_v*d_v][d_model] output gate                         */
+  const void* o_norm_w;    /* [d_v]                                                  */
+  const void* w_o;         /* [d_model][H_v*d_v] output projection                   */
+  const void* mlp_norm_w;  /* [d_model], or NULL: the block has no MLP               */
+  const void* w_gate;      /* [d_ff][d_model]                                        */
+  const void* w_up;        /* [d_ff][d_model]                                        */
+  const void* w_down;      /* [d_model][d_ff]                                        */
+  int32_t d_ff;            /* a multiple of 64; 0 without an MLP                     */
+} sr_block_weights;
+
+/* Scratch bytes sr_replay_group_states needs for the bounds in `table` and MLPs up to `max_d_ff` wide. */
+int sr_group_workspace_bytes(const sr_ctx* ctx, const sr_page_table* table, int32_t max_d_ff, size_t* out_bytes);
+
+/*
+ * Rebuilds the recurrent and conv state of layers first_layer .. first_layer + n_group_layers - 1 for every request
+ * from the group-entry anchors alone.  `weights` and `blocks`: HOST arrays with n_layers entries (the group's are
+ * read; the last layer's block needs only norm_w: its output is never formed).  Outputs, addressing, the batch
+ * table, device-side validation and status bits as in sr_replay_states; every layer of the group is written.
+ * bf16 weights (SR_W_BF16) and (d_k, d_v) in {(64, 64), (128, 128)}, d_model and H_v*d_v multiples of 64;
+ * else SR_ERR_UNSUPPORTED_SHAPE.  `debug_rows`: NULL, or DEVICE bf16 [n_group_layers - 1][max_slots * 64][d_model]
+ * receiving the rows handed from each layer to the next in packed page-slot order (request i's rows start at page
+ * slot sum_{i' < i} ceil(R_i' / 64)); a test aid.  Asynchronous on `stream`, no allocation, no host sync.
+ */
+int sr_replay_group_states(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* table,
+                           const int32_t* replay_lens, int32_t first_layer, int32_t n_group_layers,
+                           const sr_layer_weights* weights, const sr_block_weights* blocks, float norm_eps,
+                           const sr_out* out_ssm, const sr_out* out_conv, void* debug_rows, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
+/*
  * The write side of the sidecar (Section 5.1, "Writing anchors": the host precomputes a
  * destination table for the step; indexed copies inside the step's graph write the selected
  * hidden states directly to their sidecar locations; unsampled positions receive a scratch
@@ -374,7 +426,8 @@ enum {
   SR_KERNEL_WEIGHT_DECODE = 4, /* e4m3 weights only: codes -> 16-bit weights before the projection */
   SR_KERNEL_CHUNK_LOCAL = 5,   /* gates, K K^T and the chunk inverse for all chunks at once (then SCAN is the chain) */
   SR_KERNEL_ANCHOR_STAGE = 6,  /* e4m3 weights only: the layer's anchors copied to fp16 (W8A16) or quantised to e4m3 (W8A8), slot order */
-  SR_KERNEL_KINDS = 7
+  SR_KERNEL_GROUP_BLOCK = 7,   /* group replay only: row norms, gate / output / MLP GEMMs and the per-token outputs */
+  SR_KERNEL_KINDS = 8
 };
 
 /* Measurement aid: while enabled, sr_replay_states brackets each of its kernel launches with

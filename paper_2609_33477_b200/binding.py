@@ -32,11 +32,12 @@ EXPORTS = (
     "sr_conv_bytes_per_layer", "sr_workspace_bytes", "sr_replay_states", "sr_replay_states_host",
     "sr_debug_gather", "sr_device_status", "sr_last_launch_count", "sr_profile_enable", "sr_profile_read",
     "sr_replay_states_noalloc", "sr_replay_states_from", "sr_anchor_write", "sr_workspace_bytes_min",
-    "sr_debug_quantise",
+    "sr_debug_quantise", "sr_group_workspace_bytes", "sr_replay_group_states",
 )
 SR_NOALLOC_SCRATCH_BYTES = 128 * 1024 * 1024
 SR_KERNEL_SCHEDULE, SR_KERNEL_PROJECTION, SR_KERNEL_CONV_TAIL, SR_KERNEL_SCAN = 0, 1, 2, 3
-KERNEL_KINDS = {"schedule": 0, "projection": 1, "conv_tail": 2, "scan": 3, "weight_decode": 4, "chunk_local": 5, "anchor_stage": 6}
+KERNEL_KINDS = {"schedule": 0, "projection": 1, "conv_tail": 2, "scan": 3, "weight_decode": 4, "chunk_local": 5, "anchor_stage": 6,
+                "group_block": 7}
 
 
 class sr_model_desc(C.Structure):
@@ -62,6 +63,12 @@ class sr_page_table(C.Structure):
     _fields_ = [("pages", C.c_void_p), ("state_slots", C.c_void_p), ("n_requests", C.c_int32),
                 ("max_pages", C.c_int32), ("max_replay_len", C.c_int32), ("max_total_rows", C.c_int64),
                 ("n_state_slots", C.c_int32)]
+
+
+class sr_block_weights(C.Structure):
+    _fields_ = [("norm_w", C.c_void_p), ("w_z", C.c_void_p), ("o_norm_w", C.c_void_p), ("w_o", C.c_void_p),
+                ("mlp_norm_w", C.c_void_p), ("w_gate", C.c_void_p), ("w_up", C.c_void_p), ("w_down", C.c_void_p),
+                ("d_ff", C.c_int32)]
 
 
 class sr_out(C.Structure):
@@ -116,6 +123,11 @@ def load() -> C.CDLL:
     lib.sr_debug_quantise.argtypes = [
         C.c_void_p, C.POINTER(sr_anchor_pool), C.POINTER(sr_page_table), C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
         C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sr_group_workspace_bytes.argtypes = [C.c_void_p, C.POINTER(sr_page_table), C.c_int32, C.POINTER(C.c_size_t)]
+    lib.sr_replay_group_states.argtypes = [
+        C.c_void_p, C.POINTER(sr_anchor_pool), C.POINTER(sr_page_table), C.c_void_p, C.c_int32, C.c_int32,
+        C.POINTER(sr_layer_weights), C.POINTER(sr_block_weights), C.c_float, C.POINTER(sr_out), C.POINTER(sr_out),
+        C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sr_device_status.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_uint32)]
     lib.sr_last_launch_count.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
     lib.sr_profile_enable.argtypes = [C.c_void_p, C.c_int]
@@ -176,6 +188,19 @@ def sr_workspace_bytes_min(ctx, table: sr_page_table) -> int:
     n = C.c_size_t()
     _check(load().sr_workspace_bytes_min(ctx, C.byref(table), C.byref(n)), "sr_workspace_bytes_min")
     return n.value
+
+
+def sr_group_workspace_bytes(ctx, table: sr_page_table, max_d_ff: int) -> int:
+    out = C.c_size_t()
+    _check(load().sr_group_workspace_bytes(ctx, C.byref(table), int(max_d_ff), C.byref(out)), "sr_group_workspace_bytes")
+    return int(out.value)
+
+
+def sr_replay_group_states(ctx, pool, table, replay_lens_ptr, first_layer, n_group_layers, weights, blocks, norm_eps,
+                           out_ssm, out_conv, debug_rows_ptr, workspace_ptr, workspace_bytes, stream_ptr) -> int:
+    return load().sr_replay_group_states(ctx, C.byref(pool), C.byref(table), replay_lens_ptr, int(first_layer),
+                                         int(n_group_layers), weights, blocks, float(norm_eps), C.byref(out_ssm),
+                                         C.byref(out_conv), debug_rows_ptr, workspace_ptr, workspace_bytes, stream_ptr)
 
 
 def sr_replay_states(ctx, pool, table, replay_lens_ptr, layer_mask, weights, out_ssm, out_conv,
@@ -345,6 +370,42 @@ class Replayer:
         if check:
             _check(st, "sr_replay_states")
         return st
+
+    def replay_group_states(self, first_layer: int = 0, n_group_layers: Optional[int] = None, norm_eps: float = 1e-6,
+                            debug_rows: bool = False, stream=None, check: bool = True):
+        """One ``sr_replay_group_states`` call: the workload's layers first_layer .. as one group, fed by the anchors of
+        the first (Section 4.1).  With ``debug_rows`` also returns the rows handed from layer to layer, bf16
+        [n_group_layers - 1, max_slots * 64, d] in packed page-slot order."""
+        wl, spec = self.wl, self.spec
+        if wl.blocks is None:
+            raise ValueError("not a group workload")
+        g = spec.n_layers - first_layer if n_group_layers is None else int(n_group_layers)
+        if not hasattr(self, "_blocks"):
+            self._blocks = (sr_block_weights * spec.n_layers)()
+            ptr = lambda t: t.data_ptr() if t is not None else None
+            for l, b in enumerate(wl.blocks):
+                self._blocks[l] = sr_block_weights(ptr(b.norm_w), ptr(b.w_z), ptr(b.o_norm_w), ptr(b.w_o), ptr(b.mlp_norm_w),
+                                                   ptr(b.w_gate), ptr(b.w_up), ptr(b.w_down),
+                                                   int(b.w_gate.shape[0]) if b.w_gate is not None else 0)
+            max_ff = max([int(b.w_gate.shape[0]) for b in wl.blocks if b.w_gate is not None] + [0])
+            self._group_ws_bytes = sr_group_workspace_bytes(self.ctx, self.table, max_ff)
+            self._group_ws = torch.empty(self._group_ws_bytes + 256, dtype=torch.uint8, device=self.device)
+            self._group_ws_ptr = (self._group_ws.data_ptr() + 255) // 256 * 256
+        rows = None
+        if debug_rows and g > 1:
+            B = self.table.n_requests
+            max_slots = (min(self.table.max_total_rows // 64 + B, B * self.table.max_pages) + 3) // 4 * 4
+            rows = torch.zeros((g - 1, max(max_slots, 4) * 64, spec.d_model), dtype=torch.bfloat16, device=self.device)
+        st = sr_replay_group_states(self.ctx, self.pool, self.table, wl.replay_lens.data_ptr(), first_layer, g, self.weights,
+                                    self._blocks, norm_eps, self._out_ssm, self._out_conv,
+                                    rows.data_ptr() if rows is not None else None, self._group_ws_ptr, self._group_ws_bytes,
+                                    self._stream_ptr(stream))
+        if check:
+            _check(st, "sr_replay_group_states")
+        return (st, rows) if debug_rows else st
+
+    def group_device_status(self, stream=None) -> int:
+        return sr_device_status(self.ctx, self._group_ws_ptr, self._stream_ptr(stream))
 
     def replay_states_from(self, in_ssm: Optional[torch.Tensor], in_conv: Optional[torch.Tensor], stream=None,
                            check: bool = True) -> int:

@@ -335,6 +335,12 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
     fused.n_gate = ctx->n_gate;
     // page slots per run of the projection's conv epilogue (the first three rows of a run are finished by the scan)
     fused.fix_mod = ctx->w8a8 ? 1 : ((d.weight_format == SR_W_E4M3_BLOCK128 && !ctx->fp16_stage) ? 2 : 4);
+    fused.x_slot_order = 0;
+    fused.with_q = 0;
+    fused.k_ch0 = 0;
+    fused.v_ch0 = ctx->n_k;
+    fused.dump_s = nullptr;
+    fused.dump_u = nullptr;
     fused.hist = nullptr;
     fused.in_ssm_layer = nullptr;
     fused.in_ssm_slot_stride = 0;

@@ -52,7 +52,8 @@ struct sr_ctx {
 // calls return cudaSuccess at once.  A failed set-up is retried by the next call.
 enum SrOnceKey {
   SR_ONCE_PROJ_FUSED = 0, SR_ONCE_PROJ_FUSED2, SR_ONCE_CHUNK_LOCAL_64, SR_ONCE_CHUNK_LOCAL_96,
-  SR_ONCE_CHUNK_LOCAL_128, SR_ONCE_CHAIN_UMMA, SR_ONCE_CONV_GEMM, SR_ONCE_KEYS
+  SR_ONCE_CHUNK_LOCAL_128, SR_ONCE_CHAIN_UMMA, SR_ONCE_CONV_GEMM, SR_ONCE_ROWS_GEMM, SR_ONCE_GROUP_OUT_64, SR_ONCE_GROUP_OUT_96,
+  SR_ONCE_GROUP_OUT_128, SR_ONCE_KEYS
 };
 cudaError_t sr_once_per_device(int key, cudaError_t (*setup)());
 // SM count of the current device (looked up once per device)
@@ -215,6 +216,16 @@ struct SrFused {
   int32_t n_kv;
   int32_t n_gate;
   int32_t fix_mod;   // page slots per projection tile along the token axis
+  // Group replay projects the query channels for every row too (the layer's outputs need them): the hand-over tiles
+  // then hold q | k | v and the conv channel of projected channel c is c itself; otherwise they hold k | v and the
+  // conv channel is n_k + c.
+  int32_t x_slot_order;   // the projection's row operand (`pool` argument) is a packed bf16 buffer in slot order
+  int32_t with_q;    // 0: k | v tiles (state-only replay), 1: q | k | v tiles
+  int32_t k_ch0;     // first key channel inside a slot's tiles (0, or n_k with the query block in front)
+  int32_t v_ch0;     // first value channel (n_k, or 2 n_k)
+  // group replay only: what the state chain leaves for the output kernel, per (slot, value head)
+  __half* dump_s;    // [slot][H_v][d_k][d_v] fp16: the state entering the chunk (not written for a request's first chunk)
+  __half* dump_u;    // [slot][H_v][d_v][64] fp16: the chunk's pseudo-values U^T, before the row factors
 };
 
 struct SrPoolView {
@@ -266,6 +277,21 @@ bool sr_proj_fused_exact_fp8_supported(const sr_ctx* ctx);
 cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_anchor_pool& pool, int32_t pool_layer,
                                  const sr_layer_weights& w, const void* decoded, const SrFused& fused, int sm_count,
                                  cudaStream_t stream);
+
+// group replay (sr_group_gemm.cu, sr_group_output.cu)
+cudaError_t sr_launch_rows_gemm(const SrSched& s, int kind, const __nv_bfloat16* a, int64_t k, const void* b, const void* b2,
+                                int32_t n, __nv_bfloat16* c, int64_t ldc, const __nv_bfloat16* residual, int64_t ldr,
+                                int sm_count, cudaStream_t stream);
+bool sr_group_output_supported(int d_k, int d_v);
+cudaError_t sr_launch_group_output(const sr_ctx* ctx, const SrSched& s, const SrFused& fused, const void* split_buf,
+                                   const __nv_bfloat16* zg, const __nv_bfloat16* o_norm_w, float norm_eps, __nv_bfloat16* y,
+                                   cudaStream_t stream);
+// conv state of every channel from the raw rows a q | k | v projection kept (group replay)
+cudaError_t sr_launch_conv_tail_from_raw(const sr_ctx* ctx, const SrSched& s, const SrFused& fused, char* out_conv_layer,
+                                         int64_t slot_stride, cudaStream_t stream);
+cudaError_t sr_launch_rmsnorm_rows(const SrSched& s, const SrPoolView& pool, int32_t pool_layer, const __nv_bfloat16* rows_in,
+                                   const __nv_bfloat16* w, float eps, int32_t d_model, __nv_bfloat16* out,
+                                   __nv_bfloat16* copy_out, cudaStream_t stream);
 
 // Conv state: last w-1 projection rows of every channel, rounded to bf16.
 int sr_conv_tail_launches(const sr_ctx* ctx, int n_requests);

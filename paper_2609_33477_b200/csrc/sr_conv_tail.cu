@@ -412,6 +412,14 @@ cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoo
   return cudaGetLastError();
 }
 
+cudaError_t sr_launch_conv_tail_from_raw(const sr_ctx* ctx, const SrSched& s, const SrFused& fused, char* out_conv_layer,
+                                         int64_t slot_stride, cudaStream_t stream) {
+  // every conv channel was projected for every row: the last rows are all in zraw (n_q = 0, n_kv = C)
+  dim3 g((unsigned)((ctx->conv_ch + 255) / 256), (unsigned)s.n_requests);
+  sr_conv_tail_kv_kernel<<<g, 256, 0, stream>>>(s, 0, ctx->conv_ch, fused.zraw, ctx->conv_ch, nullptr, out_conv_layer, slot_stride);
+  return cudaGetLastError();
+}
+
 cudaError_t sr_launch_hist_gather(const sr_ctx* ctx, const SrSched& s, const char* in_conv_layer, int64_t slot_stride,
                                   __nv_bfloat16* hist, cudaStream_t stream) {
   const int n_vals = ctx->conv_ch * (SR_CONV_W - 1);

@@ -58,6 +58,7 @@ struct FusedParams {
   const __nv_bfloat16* hist;   // conv state each request continues from, [request][C][3], or null
   int32_t conv_ch;
   int32_t fp16_stage;    // operands are the fp16 staging copies: fp16 MMA formats, anchors in slot order (page = slot)
+  int32_t slot_order;    // the row operand is a packed buffer in slot order (page = slot), bf16 (group replay)
   int32_t group_t;       // token tiles per rasterisation group
   int32_t group_c;       // channel tiles (pair tiles in the two-CTA form) per block inside a group
 };
@@ -198,7 +199,7 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         tile_coords(tile, ct, tt);
         int page[SLOTS];
 #pragma unroll
-        for (int q = 0; q < SLOTS; ++q) page[q] = p.fp16_stage ? SLOTS * tt + q : p.s.slot_page[SLOTS * tt + q];
+        for (int q = 0; q < SLOTS; ++q) page[q] = (p.fp16_stage || p.slot_order) ? SLOTS * tt + q : p.s.slot_page[SLOTS * tt + q];
         const bool gate = ct == p.n_ct;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
@@ -614,8 +615,9 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         int pt, tt;
         tile_coords(tile, pt, tt);
         const int slot_a = SLOTS * tt + 2 * rank;
-        int page0 = p.fp16_stage ? slot_a : p.s.slot_page[slot_a], page1 = p.fp16_stage ? slot_a + 1 : p.s.slot_page[slot_a + 1];
-        if (!p.fp16_stage && p.s.check_bounds) {      // a bad page id would only read the fill value (TMA clips), but say so
+        const bool by_slot = p.fp16_stage || p.slot_order;
+        int page0 = by_slot ? slot_a : p.s.slot_page[slot_a], page1 = by_slot ? slot_a + 1 : p.s.slot_page[slot_a + 1];
+        if (!by_slot && p.s.check_bounds) {      // a bad page id would only read the fill value (TMA clips), but say so
           if (!sr_check_page(p.s, page0)) page0 = 0;
           if (!sr_check_page(p.s, page1)) page1 = 0;
         }
@@ -736,7 +738,10 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   if (stage && (!fused.x16 || !fused.w16)) return cudaErrorInvalidValue;
   if (a8 && (!fused.x8 || !fused.sx)) return cudaErrorInvalidValue;
   const int d = ctx->desc.d_model;
-  const int n_kv = ctx->n_k + ctx->n_v;
+  // channels this launch projects: k | v, or q | k | v for group replay (bf16 weights only)
+  if (fused.with_q && (stage || a8 || scaled)) return cudaErrorInvalidValue;
+  const int n_kv = fused.with_q ? ctx->conv_ch : ctx->n_k + ctx->n_v;
+  const int ch0 = fused.with_q ? 0 : ctx->n_k;          // row of W_qkv / conv channel of projected channel 0
   CUtensorMap map_x, map_w, map_g;
   if (stage) {
     sr_anchor_pool staged = pool;                       // the layer's anchors in slot order: "page" = slot
@@ -764,11 +769,12 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   p.s = s;
   p.pool_layer = stage ? 0 : pool_layer;
   p.fp16_stage = stage;
+  p.slot_order = fused.x_slot_order;
   p.hist = fused.hist;
   p.conv_ch = ctx->conv_ch;
   p.k_blocks = d / BK;
-  p.n_q = ctx->n_k;
-  p.w_row0 = (scaled || stage) ? 0 : ctx->n_k;
+  p.n_q = ch0;
+  p.w_row0 = (scaled || stage) ? 0 : ch0;
   p.n_ct = (n_kv + BM - 1) / BM;
   p.n_gate = ctx->n_gate;
   p.ncb = fused.ncb;

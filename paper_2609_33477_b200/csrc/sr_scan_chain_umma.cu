@@ -39,7 +39,7 @@ namespace {
 constexpr int CH = 64;
 constexpr int D = 128;                   // tile height and MMA M: head widths up to 128 per CTA
 constexpr int TT_HALFS = 2 * CH * CH;
-constexpr int SC_FLOATS = 128;
+constexpr int SC_FLOATS = 256;
 constexpr int COMPUTE_THREADS = 256;
 constexpr int THREADS = COMPUTE_THREADS + 32;
 constexpr int TILE_KV = D * CH * 2;      // 16 KB: [128][64] fp16
@@ -75,6 +75,9 @@ struct ChainUmmaParams {
   int32_t erase;             // 0: decay-only family, U = U~ (no W S term)
   const char* in_layer;      // states to continue from (same slot addressing as the output), or null = zero
   int64_t in_slot_stride;
+  int32_t k_ch0, v_ch0;      // first key / value channel inside a slot's tiles
+  __half* dump_s;            // group replay: [slot][H_v][d_k][d_v] state entering each chunk (fp16), or null
+  __half* dump_u;            // group replay: [slot][H_v][d_v][64] pseudo-values of each chunk (fp16), or null
   long long wait_limit;      // cycles a wait may take before it gives up
   int32_t withhold_first_keys;   // fault injection (SR_DEBUG_EXPIRE_WAIT): chunk 0's key tile is never requested, so
                                  // the waits on it run out
@@ -168,7 +171,7 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
   // tile rows in the tensor maps: channel c of slot s is row s * (ncb * 128) + c (keys of key head a from
   // a * d_k, values of value head h from H_k d_k + h * d_v), 128 rows fetched whatever the head width;
   // T matrices of (slot, head) start at row (slot*H_v + head)*128 (Tb), +64 (Tw)
-  const int k_row = kh * dk, v_row = p.n_k_heads * dk + h * dv + col0, slot_rows = p.ncb * D;
+  const int k_row = p.k_ch0 + kh * dk, v_row = p.v_ch0 + h * dv + col0, slot_rows = p.ncb * D;
   auto load_v = [&](int ck) {          // V^T, Tb, Tw of chunk ck (one buffer)
     const int slot = slot0 + ck;
     uint64_t* bar = &sm.bar_v[ck & 1];
@@ -284,6 +287,14 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
             float v[32];
             tmem_ld32(tm_S + lane_off + (uint32_t)(half * 64 + c * 32), v);
             if (erase) store_row32(sm.S16 + half * TILE_KV, row, c * 32, v);
+            if (p.dump_s && row < dk) {          // the state entering this chunk, for the layer's per-token outputs
+              __half* ds = p.dump_s + (((long long)(slot0 + ck) * p.n_v_heads + h) * dk + row) * dv + col0 + half * 64 + c * 32;
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                if (half * 64 + c * 32 + 8 * q < dvb)
+                  *(uint4*)(ds + 8 * q) = make_uint4(pack_h2(v[8 * q], v[8 * q + 1]), pack_h2(v[8 * q + 2], v[8 * q + 3]),
+                                                     pack_h2(v[8 * q + 4], v[8 * q + 5]), pack_h2(v[8 * q + 6], v[8 * q + 7]));
+            }
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] *= decay;
             tmem_st32(tm_S + lane_off + (uint32_t)(half * 64 + c * 32), v);
@@ -309,6 +320,13 @@ sr_scan_chain_umma_kernel(const __grid_constant__ CUtensorMap map_kv, const __gr
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         float v[32];
         tmem_ld32(tm_U + lane_off + (uint32_t)(half * 32), v);
+        if (p.dump_u && row < dvb) {             // U^T of this chunk: value index `row`, chunk rows half * 32 ..
+          __half* du = p.dump_u + (((long long)(slot0 + ck) * p.n_v_heads + h) * dv + col0 + row) * CH + half * 32;
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            *(uint4*)(du + 8 * q) = make_uint4(pack_h2(v[8 * q], v[8 * q + 1]), pack_h2(v[8 * q + 2], v[8 * q + 3]),
+                                               pack_h2(v[8 * q + 4], v[8 * q + 5]), pack_h2(v[8 * q + 6], v[8 * q + 7]));
+        }
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] *= sc[half * 32 + i];              // f_j of chunk row j
         store_row32(sm.WU, row, half * 32, v);
@@ -396,6 +414,10 @@ cudaError_t sr_launch_scan_chain_umma(const sr_ctx* ctx, const SrSched& s, const
   p.out_layer = out_ssm_layer;
   p.slot_stride = slot_stride;
   p.erase = d.recurrence == SR_REC_GATED_DELTA;
+  p.k_ch0 = fused.k_ch0;
+  p.v_ch0 = fused.v_ch0;
+  p.dump_s = fused.dump_s;
+  p.dump_u = fused.dump_u;
   p.in_layer = fused.in_ssm_layer;
   p.in_slot_stride = fused.in_ssm_slot_stride;
   p.withhold_first_keys = (ctx->debug_flags & SR_DEBUG_EXPIRE_WAIT) ? 1 : 0;

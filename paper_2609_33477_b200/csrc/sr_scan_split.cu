@@ -26,7 +26,8 @@ constexpr int CH = 64;            // chunk rows (= page rows)
 constexpr int LDT = CH + 8;       // pitch (halfs) of 64 x 64 fp16 tiles
 constexpr int LDK = CH + 8;       // pitch (halfs) of channel-major [d_k][64] key tiles
 constexpr int TT_HALFS = 2 * CH * CH;   // per chunk and head: T diag(beta), then T diag(beta gamma n)
-constexpr int SC_FLOATS = 128;          // per chunk and head: 64 row factors, gamma_n, padding
+constexpr int SC_FLOATS = 256;          // per chunk and head: 64 row factors, gamma_n, padding | 64 running log-decays g_i |
+                                        // 64 inverse key norms
 
 // ---------------------------------------------------------------------------------------------------
 // chunk-local part
@@ -62,6 +63,8 @@ struct LocalParams {
   int32_t ncb, n_kv, fix_mod;
   int32_t n_k_heads, n_v_heads;
   int32_t d_v;                    // value head width (the key head width is the template parameter)
+  int32_t with_q, k_ch0, v_ch0;   // tile contents (see SrFused); conv channel of projected channel c = conv_ch0 + c
+  int32_t conv_ch0;
   int32_t act_identity;
   int32_t erase;                  // 0: decay-only family, A = 0 and T = I
   float eps;
@@ -108,8 +111,10 @@ __global__ void __launch_bounds__(LT, LOCAL_CTAS_PER_SM) sr_chunk_local_kernel(c
   const int n_k = p.n_k_heads * DK, dv = p.d_v;
   const bool fix = !p.s.slot_first[slot] && (slot % p.fix_mod) == 0;
   const long long slot_ch = (long long)slot * p.ncb * 128;        // first channel row of this slot's tiles
-  __half* tk = p.kv16 + (slot_ch + kh * DK) * CH;
-  __half* tv = p.kv16 + (slot_ch + n_k + h * dv) * CH;
+  __half* tk = p.kv16 + (slot_ch + p.k_ch0 + kh * DK) * CH;
+  __half* tv = p.kv16 + (slot_ch + p.v_ch0 + h * dv) * CH;
+  __half* tq = p.kv16 + (slot_ch + kh * DK) * CH;                  // with_q only: the key head's query channels
+  const int qn = p.with_q ? DK : 0;                                // fix-up channels: [q |] k | v of this head
 
   // ---- fetch: the key tile and the two gate rows of this head ----
   for (int i = tid; i < DK * (CH / 8); i += LT) {
@@ -124,14 +129,16 @@ __global__ void __launch_bounds__(LT, LOCAL_CTAS_PER_SM) sr_chunk_local_kernel(c
   asm volatile("cp.async.commit_group;" ::: "memory");
   // where a fix-up is due: the previous slot's last three raw rows and this slot's rows 0..2 of this thread's
   // channels (the head's d_k key channels, then its d_v value channels), fetched while the key tile is in flight
-  constexpr int FIXQ = 3;         // channels per thread: d_k + d_v <= 3 * 128
+  constexpr int FIXQ = 4;         // channels per thread: (d_k +) d_k + d_v <= 4 * 128
   float zr[FIXQ][6];
+  // channel c of the head's run -> its index among the projected channels
+  auto run_channel = [&](int c) { return c < qn ? kh * DK + c : (c < qn + DK ? p.k_ch0 + kh * DK + (c - qn) : p.v_ch0 + h * dv + (c - qn - DK)); };
   if (fix) {
 #pragma unroll
     for (int q = 0; q < FIXQ; ++q) {
       const int c = tid + q * LT;
-      if (c < DK + dv) {
-        const int zc = c < DK ? kh * DK + c : n_k + h * dv + (c - DK);
+      if (c < qn + DK + dv) {
+        const int zc = run_channel(c);
 #pragma unroll
         for (int rr = 0; rr < 6; ++rr)
           zr[q][rr] = __ldg(p.zraw + ((long long)(rr < 3 ? slot - 1 : slot) * 6 + (rr < 3 ? 3 + rr : rr - 3)) * p.n_kv + zc);
@@ -147,20 +154,20 @@ __global__ void __launch_bounds__(LT, LOCAL_CTAS_PER_SM) sr_chunk_local_kernel(c
 #pragma unroll
     for (int q = 0; q < FIXQ; ++q) {
       const int c = tid + q * LT;
-      if (c < DK + dv) {
-        const int zc = c < DK ? kh * DK + c : n_k + h * dv + (c - DK);
-        const uint2 wv = *(const uint2*)(p.conv_w + (long long)(n_k + zc) * SR_CONV_W);
+      if (c < qn + DK + dv) {
+        const int zc = run_channel(c);
+        const uint2 wv = *(const uint2*)(p.conv_w + (long long)(p.conv_ch0 + zc) * SR_CONV_W);
         const __nv_bfloat16* e = (const __nv_bfloat16*)&wv;
         const float w0 = __bfloat162float(e[0]), w1 = __bfloat162float(e[1]), w2 = __bfloat162float(e[2]),
                     w3 = __bfloat162float(e[3]);
-        __half* gdst = c < DK ? tk + c * CH : tv + (c - DK) * CH;
+        __half* gdst = c < qn ? tq + c * CH : (c < qn + DK ? tk + (c - qn) * CH : tv + (c - qn - DK) * CH);
 #pragma unroll
         for (int rho = 0; rho < 3; ++rho) {
           float y = w0 * zr[q][rho] + w1 * zr[q][rho + 1] + w2 * zr[q][rho + 2] + w3 * zr[q][rho + 3];
           if (!p.act_identity) y = __fdividef(y, 1.f + __expf(-y));
           const __half hy = __float2half_rn(y);
           gdst[rho] = hy;
-          if (c < DK) sm.Ks[c * LDK + rho] = hy;
+          if (c >= qn && c < qn + DK) sm.Ks[(c - qn) * LDK + rho] = hy;
         }
       }
     }
@@ -401,6 +408,10 @@ __global__ void __launch_bounds__(LT, LOCAL_CTAS_PER_SM) sr_chunk_local_kernel(c
     const float g_last = sm.g[CH - 1];
     float* sc = p.sc + ((long long)slot * p.n_v_heads + h) * SC_FLOATS;
     sc[tid] = tid < CH ? __expf(g_last - sm.g[tid]) * sm.ninv[tid] : __expf(g_last);
+    if (tid < CH) {                 // for the output kernel of group replay
+      sc[128 + tid] = sm.g[tid];
+      sc[192 + tid] = sm.ninv[tid];
+    }
   }
 }
 
@@ -411,7 +422,7 @@ size_t sr_scan_split_bytes(const sr_ctx* ctx, int64_t max_slots) {
 }
 
 bool sr_chunk_local_supported(int d_k, int d_v) {
-  return (d_k == 64 || d_k == 96 || d_k == 128) && d_v % 8 == 0 && d_v > 0 && d_k + d_v <= 3 * LT;
+  return (d_k == 64 || d_k == 96 || d_k == 128) && d_v % 8 == 0 && d_v > 0 && 2 * d_k + d_v <= 4 * LT;
 }
 
 template <int DK>
@@ -439,6 +450,10 @@ cudaError_t sr_launch_chunk_local(const sr_ctx* ctx, const SrSched& s, const sr_
   p.n_k_heads = d.n_k_heads;
   p.n_v_heads = d.n_v_heads;
   p.d_v = d.d_v;
+  p.with_q = fused.with_q;
+  p.k_ch0 = fused.k_ch0;
+  p.v_ch0 = fused.v_ch0;
+  p.conv_ch0 = fused.with_q ? 0 : ctx->n_k;
   p.act_identity = d.conv_activation == SR_CONV_IDENTITY;
   p.erase = d.recurrence == SR_REC_GATED_DELTA;
   p.eps = d.l2_eps;

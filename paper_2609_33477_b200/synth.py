@@ -52,6 +52,10 @@ class WorkloadSpec:
     n_trunks: int = 16                # "trunks" paging only
     trunk_pages: int = 256            # "trunks" paging only
     requests_per_trunk: int = 4       # "trunks" paging only
+    # group-propagated replay (Section 4.1): all n_layers form ONE group of consecutive linear-attention layers whose
+    # only anchors are the rows entering layer 0; every layer gets block weights, and an MLP d_ff[l] wide (0: none)
+    group: bool = False
+    d_ff: Tuple = ()
 
     @property
     def conv_channels(self) -> int:
@@ -135,6 +139,16 @@ SPECS["cfg4_w8a8_slice"] = dataclasses.replace(SPECS["cfg4_slice"], name="cfg4_w
 SPECS["w8a8_small"] = dataclasses.replace(SPECS["fp8_small"], name="w8a8_small", act_quant="e4m3_1x128")
 SPECS["w8a8_ragged"] = _spec("w8a8_ragged", 2, 1024, 4, 128, 5, ("list", (0, 3, 65, 200, 700)), weight_format="e4m3_block128",
                              act_quant="e4m3_1x128", layer_mask="even")
+# Group-propagated replay: small cases per supported geometry (ragged lengths, an empty request, MLP on some layers)
+# and the 4B geometry with three linear-attention layers per group (the 3 : 1 hybrid pattern), eight 512-row hits.
+SPECS["group_small"] = WorkloadSpec(name="group_small", n_layers=3, d_model=256, n_k_heads=2, n_v_heads=4, d_k=64, d_v=64,
+                                    n_requests=4, replay=("list", (0, 70, 200, 130)), group=True, d_ff=(0, 192, 0))
+SPECS["group_128"] = WorkloadSpec(name="group_128", n_layers=2, d_model=512, n_k_heads=2, n_v_heads=4, d_k=128, d_v=128,
+                                  n_requests=2, replay=("list", (300, 64)), group=True, d_ff=(512, 0))
+SPECS["group_wide"] = WorkloadSpec(name="group_wide", n_layers=2, d_model=640, n_k_heads=1, n_v_heads=3, d_k=128, d_v=128,
+                                   n_requests=3, replay=("list", (129, 1, 257)), group=True, d_ff=(448, 0))
+SPECS["group3_4b"] = WorkloadSpec(name="group3_4b", n_layers=3, d_model=2560, n_k_heads=16, n_v_heads=32, d_k=128, d_v=128,
+                                  n_requests=8, replay=("fixed", 512), group=True, d_ff=(10240, 10240, 10240))
 for _r in (1024, 2048, 4096):
     SPECS[f"cfg4_R{_r}"] = dataclasses.replace(SPECS["cfg4"], name=f"cfg4_R{_r}", replay=("fixed", _r))
 
@@ -151,6 +165,19 @@ class LayerParams:
 
 
 @dataclasses.dataclass
+class BlockParams:
+    """The rest of one block of a group (Section 4.1): norms, output gate and projection, optional MLP.  All bf16."""
+    norm_w: torch.Tensor                # [d]
+    w_z: torch.Tensor                   # [H_v d_v, d]
+    o_norm_w: torch.Tensor              # [d_v]
+    w_o: torch.Tensor                   # [d, H_v d_v]
+    mlp_norm_w: Optional[torch.Tensor] = None   # [d]
+    w_gate: Optional[torch.Tensor] = None       # [f, d]
+    w_up: Optional[torch.Tensor] = None         # [f, d]
+    w_down: Optional[torch.Tensor] = None       # [d, f]
+
+
+@dataclasses.dataclass
 class Workload:
     spec: WorkloadSpec
     anchor_pool: torch.Tensor           # [n_phys, L_pool, PAGE_ROWS, d] bf16
@@ -159,6 +186,7 @@ class Workload:
     page_table: torch.Tensor            # [B, max_pages] int32, oldest page first, -1 padding
     replay_lens: torch.Tensor           # [B] int32, rows to replay per request
     layers: List[Optional[LayerParams]]  # None for masked-out layers
+    blocks: Optional[List[BlockParams]] = None   # group workloads only
 
     @property
     def n_phys_pages(self) -> int:
@@ -273,7 +301,10 @@ def build_workload(spec_or_name, device="cpu", seed: int = 0,
         raise ValueError(spec.layer_mask)
     layer_to_pool, n_pool = [], 0
     for l in range(spec.n_layers):
-        if mask[l]:
+        if spec.group:                 # one anchor per group: the rows entering its first layer
+            layer_to_pool.append(0 if l == 0 else -1)
+            n_pool = 1
+        elif mask[l]:
             layer_to_pool.append(n_pool)
             n_pool += 1
         else:
@@ -310,9 +341,31 @@ def build_workload(spec_or_name, device="cpu", seed: int = 0,
             decay_scale=torch.full((Hv,), spec.decay_scale, dtype=torch.float32, device=device),
             dt_bias=torch.zeros((Hv,), dtype=torch.float32, device=device)))
 
+    blocks = None
+    if spec.group:
+        hv = Hv * spec.d_v
+        blocks = []
+
+        def uniform(n, tid, l):        # norm weights around 1
+            g = _generator(device, seed, tid, l)
+            return (0.5 + torch.rand(n, generator=g, device=device, dtype=torch.float32)).to(torch.bfloat16)
+
+        for l in range(spec.n_layers):
+            b = BlockParams(norm_w=uniform(d, 6, l),
+                            w_z=_normal((hv, d), d ** -0.5, _generator(device, seed, 7, l), device, torch.bfloat16),
+                            o_norm_w=uniform(spec.d_v, 8, l),
+                            w_o=_normal((d, hv), hv ** -0.5, _generator(device, seed, 9, l), device, torch.bfloat16))
+            f = spec.d_ff[l] if l < len(spec.d_ff) else 0
+            if f:
+                b.mlp_norm_w = uniform(d, 10, l)
+                b.w_gate = _normal((f, d), d ** -0.5, _generator(device, seed, 11, l), device, torch.bfloat16)
+                b.w_up = _normal((f, d), d ** -0.5, _generator(device, seed, 12, l), device, torch.bfloat16)
+                b.w_down = _normal((d, f), f ** -0.5, _generator(device, seed, 13, l), device, torch.bfloat16)
+            blocks.append(b)
+
     return Workload(spec=spec, anchor_pool=pool, layer_to_pool=layer_to_pool, layer_mask=mask,
                     page_table=torch.from_numpy(table).to(device),
-                    replay_lens=torch.from_numpy(lens).to(device), layers=layers)
+                    replay_lens=torch.from_numpy(lens).to(device), layers=layers, blocks=blocks)
 
 
 # ---- raw-byte views for the CPU side -------------------------------------------------
@@ -336,6 +389,16 @@ def layer_arrays(p: LayerParams) -> dict:
     else:
         out["w_qkv_codes"] = p.w_qkv.detach().cpu().numpy().astype(np.uint8)
         out["w_qkv_scale"] = p.w_qkv_scale.detach().cpu().numpy().astype(np.float32)
+    return out
+
+
+def block_arrays(p: LayerParams, b: BlockParams) -> dict:
+    """One group layer's parameters as fp64 arrays of the stored values (exact: bf16 -> fp64 loses nothing)."""
+    f64 = lambda t: t.detach().to(torch.float64).cpu().numpy()
+    out = dict(norm_w=f64(b.norm_w), w_qkv=f64(p.w_qkv), w_ab=f64(p.w_ab), conv_w=f64(p.conv_w),
+               decay_scale=f64(p.decay_scale), dt_bias=f64(p.dt_bias), w_z=f64(b.w_z), o_norm_w=f64(b.o_norm_w), w_o=f64(b.w_o))
+    if b.mlp_norm_w is not None:
+        out.update(mlp_norm_w=f64(b.mlp_norm_w), w_gate=f64(b.w_gate), w_up=f64(b.w_up), w_down=f64(b.w_down))
     return out
 
 

@@ -130,3 +130,29 @@ def test_status_strings(lib):
     assert lib.sr_status_string(0) == b"SR_OK"
     assert lib.sr_status_string(B.SR_ERR_WORKSPACE) == b"SR_ERR_WORKSPACE"
     assert lib.sr_status_string(99) == b"SR_ERR_UNKNOWN"
+
+
+def test_group_replay_checks_its_arguments_on_the_host(lib):
+    """Section 4.1 entry: geometry, weight format, group range and null pointers are refused before any launch."""
+    n = C.c_size_t()
+    table = B.sr_page_table(None, None, 3, 4, 256, 600)
+    ctx = B.sr_create(_desc())
+    assert lib.sr_group_workspace_bytes(None, C.byref(table), 0, C.byref(n)) == B.SR_ERR_INVALID_ARG
+    assert lib.sr_group_workspace_bytes(ctx, C.byref(table), -64, C.byref(n)) == B.SR_ERR_INVALID_ARG
+    plain = B.sr_group_workspace_bytes(ctx, table, 0)
+    wide = B.sr_group_workspace_bytes(ctx, table, 1024)
+    assert wide - plain >= 12 * 64 * 1024 * 2 and plain > B.sr_workspace_bytes_min(ctx, table)   # the MLP's hidden rows
+    pool, out = B.sr_anchor_pool(), B.sr_out()
+    weights, blocks = (B.sr_layer_weights * 2)(), (B.sr_block_weights * 2)()
+    args = (C.byref(pool), C.byref(table), None)
+    tail = (weights, blocks, C.c_float(1e-6), C.byref(out), C.byref(out), None, None, 0, None)
+    assert lib.sr_replay_group_states(ctx, *args, 0, 2, *tail) == B.SR_ERR_INVALID_ARG      # null pointers
+    assert lib.sr_replay_group_states(None, *args, 0, 2, *tail) == B.SR_ERR_INVALID_ARG
+    B.sr_destroy(ctx)
+    fp8 = B.sr_create(_desc(weight_format=B.SR_W_E4M3_BLOCK128))       # block-scaled weights: single-layer replay only
+    assert lib.sr_group_workspace_bytes(fp8, C.byref(table), 0, C.byref(n)) == B.SR_ERR_UNSUPPORTED_SHAPE
+    B.sr_destroy(fp8)
+    odd = B.sr_create(_desc(d_k=96, d_v=192, n_k_heads=2, n_v_heads=2))   # replayable, but no per-token output kernel
+    assert lib.sr_workspace_bytes(odd, C.byref(table), C.byref(n)) == B.SR_OK
+    assert lib.sr_group_workspace_bytes(odd, C.byref(table), 0, C.byref(n)) == B.SR_ERR_UNSUPPORTED_SHAPE
+    B.sr_destroy(odd)
