@@ -133,7 +133,10 @@ static inline SrWorkspace sr_workspace_layout(const sr_ctx* ctx, int32_t n_reque
 
 // Layers in flight at once for a batch of these bounds: as many (up to SR_MAX_LANES, and no more than the model has
 // layers) as keep the hand-over buffers together within SR_LANES_BUDGET_BYTES; large batches fill the device with
-// one layer and get one lane.
+// one layer and get one lane.  (Measured with a 24 GiB budget, i.e. two to four lanes on the 250 000-row
+// configurations, in the same run as one lane: the chunk-local kernel does run in the shared memory the next
+// layer's persistent projection leaves free, but the projection slows by as much -- steps 1.8 % and 1.0 % shorter
+// on two configurations, 1.1 % longer on the third.)
 static inline int sr_policy_lanes(const sr_ctx* ctx, int32_t n_requests, int32_t max_pages, int64_t max_total_rows) {
   const size_t per_lane = sr_workspace_layout(ctx, n_requests, max_pages, max_total_rows, 1).lane_bytes;
   int lanes = SR_MAX_LANES;
