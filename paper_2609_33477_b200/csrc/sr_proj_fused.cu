@@ -335,26 +335,26 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 // order), tcgen05 kind::f8f6f4, one 128-byte row of K per stage.  Both operands carry block scales that are plain
 // fp32 numbers, not the hardware's power-of-two block format, so every 128-deep K group has to enter the result as
 //     total[channel][token] += w_scale[channel block][group] * x_scale[token][group] * partial[channel][token]
-// outside the tensor core.  Keeping `total` in registers (128 values per epilogue thread) spills; here it lives in
-// tensor memory next to the partial sums: columns 0..127 and 128..255 hold the partial sums of the tile's two token
-// halves (each half its own MMA of N = 128 and its own full / empty barriers, so the halves pipeline against each
-// other), columns 256..511 hold the totals.  An epilogue warp owns 32 lanes x 64 columns of each half: it loads a
-// chunk of partial sums and the matching chunk of totals, does the multiply-add with the scale products shared
-// through shared memory, and stores the totals back.  After the last group the same warp runs the conv + SiLU
-// epilogue on its two page slots (slots hw and hw + 2 of the tile's four: their conv history lies with another
-// warp, so every slot's first three rows are finished later, like the first rows of a tile in the 16-bit kernels).
+// outside the tensor core: one multiply-add per output element per group, which is what bounds this kernel.
+// Layout: three warpgroups.  Warpgroup 0 holds the TMA producer and the MMA issuer and gives most of its registers
+// away (setmaxnreg); warpgroups 1 and 2 take them and keep the TOTALS IN REGISTERS -- a thread owns one channel
+// (tensor-memory lane) and 128 tokens, warpgroup 1 the tile's first two page slots, warpgroup 2 the other two.  The
+// partial sums of a group (128 channels x 256 tokens, one MMA of N = 256 per 32 codes of K) are double-buffered in
+// tensor memory (2 x 256 columns), so the tensor core works on group g + 1 while the warpgroups fold group g.  After
+// the last group the conv + SiLU epilogue runs straight from the registers (every slot's first three rows are
+// finished later by the chunk-local kernel, like the first rows of a tile in the 16-bit kernels).
 constexpr int W8_BK = 128;                       // bytes (= codes) of K per stage
-constexpr int W8_NH = BN / 2;                    // tokens per half tile
+constexpr int W8_THREADS = 384;
 constexpr int W8_SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + 2 * 2 * BN * 4;
 
-__global__ void __launch_bounds__(NUM_THREADS_SCALED, 1)
+__global__ void __launch_bounds__(W8_THREADS, 1)
 sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const FusedParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* full_bar = (uint64_t*)(smem + STAGES * STAGE_BYTES);
   uint64_t* empty_bar = full_bar + STAGES;
-  uint64_t* pfull_bar = empty_bar + STAGES;      // [2] partial sums of a token half complete
-  uint64_t* pempty_bar = pfull_bar + 2;          // [2] ... drained by the eight epilogue warps
+  uint64_t* pfull_bar = empty_bar + STAGES;      // [2] partial sums of a group complete in buffer b
+  uint64_t* pempty_bar = pfull_bar + 2;          // [2] ... folded into the totals by the eight epilogue warps
   uint64_t* sx_full = pempty_bar + 2;            // [2] activation scales of a K group landed
   uint32_t* tmem_slot = (uint32_t*)(sx_full + 2);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
@@ -396,8 +396,9 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     tt = g * p.group_t + r / gc;
   };
 
-  if (warp == 0) {
-    if (lane == 0) {                             // TMA producer
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    if (warp == 0 && lane == 0) {                // TMA producer
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -416,54 +417,44 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-    }
-  } else if (warp == 1) {
-    if (lane == 0) {                             // MMA issue
+    } else if (warp == 1 && lane == 0) {         // MMA issue
       int stage = 0;
       uint32_t phase = 0, gcount = 0;
       bool ok = true;
-      const uint32_t idesc = umma_idesc_e4m3(BM, W8_NH);
+      const uint32_t idesc = umma_idesc_e4m3(BM, BN);
       for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
         int ct, tt;
         tile_coords(tile, ct, tt);
-        for (int kg = 0; ok && kg < k_groups; ++kg, ++gcount) {
-          const uint32_t b = gcount & 1u, par = (gcount >> 1) & 1u;
-          for (int h = 0; h < 2; ++h) {
-            // the epilogue has drained this half's partial sums of the previous group
-            if (!mbar_wait(&pempty_bar[h], ((gcount & 1u) ^ 1u), abort_flag, p.s.status)) { ok = false; break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (h == 0) {
-              // ... which also means the group before that is finished everywhere: its scale buffer is free.  Fetch this
-              // group's activation scales (one 64-float run per page slot) while the MMAs run.
-              mbar_expect_tx(&sx_full[b], BN * 4);
+        for (int kg = 0; kg < k_groups; ++kg, ++gcount) {
+          const uint32_t b = gcount & 1u;
+          // buffer b was folded two groups ago: its partial sums and its scale buffer are free
+          if (!mbar_wait(&pempty_bar[b], ((gcount >> 1) & 1u) ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          mbar_expect_tx(&sx_full[b], BN * 4);   // this group's activation scales: one 64-float run per page slot
 #pragma unroll
-              for (int q = 0; q < SLOTS; ++q)
-                bulk_load(sxs + b * BN + q * SR_PAGE_ROWS, p.sx + ((long long)(SLOTS * tt + q) * k_groups + kg) * SR_PAGE_ROWS,
-                          SR_PAGE_ROWS * 4, &sx_full[b]);
-              if (!mbar_wait(&full_bar[stage], phase, abort_flag, p.s.status)) { ok = false; break; }
-              asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            }
-            const uint32_t a_addr = smem_u32(smem + stage * STAGE_BYTES);
-            const uint64_t a_desc = umma_smem_desc(a_addr);
-            const uint64_t b_desc = umma_smem_desc(a_addr + A_BYTES + h * (B_BYTES / 2));
+          for (int q = 0; q < SLOTS; ++q)
+            bulk_load(sxs + b * BN + q * SR_PAGE_ROWS, p.sx + ((long long)(SLOTS * tt + q) * k_groups + kg) * SR_PAGE_ROWS,
+                      SR_PAGE_ROWS * 4, &sx_full[b]);
+          if (!mbar_wait(&full_bar[stage], phase, abort_flag, p.s.status)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a_addr = smem_u32(smem + stage * STAGE_BYTES);
+          const uint64_t a_desc = umma_smem_desc(a_addr), b_desc = umma_smem_desc(a_addr + A_BYTES);
 #pragma unroll
-            for (int k = 0; k < W8_BK / 32; ++k)
-              umma_e4m3(tmem_base + (uint32_t)(h * W8_NH), a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, k != 0 ? 1u : 0u);
-            umma_commit(&pfull_bar[h]);
-          }
-          (void)par;
-          if (!ok) break;
-          umma_commit(&empty_bar[stage]);        // the stage is free once both halves' products have read it
+          for (int k = 0; k < W8_BK / 32; ++k)
+            umma_e4m3(tmem_base + b * (uint32_t)BN, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, k != 0 ? 1u : 0u);
+          umma_commit(&pfull_bar[b]);
+          umma_commit(&empty_bar[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else {
-    // epilogue: tensor-memory lanes 32 * (warp % 4) .., columns hw * 64 .. of each token half
-    const int quarter = warp & 3, hw = (warp - 2) >> 2;
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+    // epilogue: tensor-memory lanes 32 * (warp % 4) .., tokens wg * 128 .. + 127 of the tile
+    const int quarter = warp & 3, wg = (warp >> 2) - 1;
     const int ch_local = quarter * 32 + lane;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    const int e = (warp - 2) * 32 + lane;        // 0..255: this thread's entry of the scale products
+    const int e = wg * 128 + (warp & 3) * 32 + lane;       // this thread's entry of the scale products
     uint32_t gcount = 0;
     bool ok = true;
     for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
@@ -471,47 +462,54 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
       tile_coords(tile, ct, tt);
       const int ch = ct * BM + ch_local;
       const float* scale_row = p.w_scale + (long long)((p.n_q + ct * BM) / 128) * p.scale_ld;
+      float tot[128];
+#pragma unroll
+      for (int i = 0; i < 128; ++i) tot[i] = 0.f;
       for (int kg = 0; kg < k_groups; ++kg, ++gcount) {
-        const uint32_t b = gcount & 1u, par_sx = (gcount >> 1) & 1u, par_p = gcount & 1u;
-        // weight scale x activation scale for the tile's 256 tokens: one product per epilogue thread
-        if (ok) ok = mbar_wait(&sx_full[b], par_sx, abort_flag, p.s.status);
+        const uint32_t b = gcount & 1u, par = (gcount >> 1) & 1u;
+        // weight scale x activation scale for this warpgroup's 128 tokens: one product per thread
+        if (ok) ok = mbar_wait(&sx_full[b], par, abort_flag, p.s.status);
         comb[b * BN + e] = ok ? __ldg(scale_row + kg) * sxs[b * BN + e] : 0.f;
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+        asm volatile("bar.sync %0, 128;" ::"r"(2 + wg) : "memory");
+        if (ok) ok = mbar_wait(&pfull_bar[b], par, abort_flag, p.s.status);
+        if (ok) {
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t col = b * (uint32_t)BN + (uint32_t)(wg * 128);
+          const float4* cb = (const float4*)(comb + b * BN + wg * 128);        // same address in every lane
+          float v0[32], v1[32];
+          tmem_ld32_issue(tmem_base + lane_off + col, v0);
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          if (ok) ok = mbar_wait(&pfull_bar[h], par_p, abort_flag, p.s.status);
-          if (ok) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t col = (uint32_t)(h * W8_NH + hw * 64);
+          for (int c = 0; c < 4; c += 2) {
+            tmem_ld32_issue(tmem_base + lane_off + col + (uint32_t)((c + 1) * 32), v1);
+            tmem_wait_ld();                      // waits for both; the second is consumed after the first chunk's math
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-              float v[32], t[32];
-              tmem_ld32_issue(tmem_base + lane_off + col + (uint32_t)(c * 32), v);
-              if (kg > 0) tmem_ld32_issue(tmem_base + lane_off + (uint32_t)BN + col + (uint32_t)(c * 32), t);
-              tmem_wait_ld();
-              const float4* cb = (const float4*)(comb + b * BN + col + c * 32);      // same address in every lane
-#pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                const float4 a = cb[q];
-                t[4 * q] = kg > 0 ? fmaf(a.x, v[4 * q], t[4 * q]) : a.x * v[4 * q];
-                t[4 * q + 1] = kg > 0 ? fmaf(a.y, v[4 * q + 1], t[4 * q + 1]) : a.y * v[4 * q + 1];
-                t[4 * q + 2] = kg > 0 ? fmaf(a.z, v[4 * q + 2], t[4 * q + 2]) : a.z * v[4 * q + 2];
-                t[4 * q + 3] = kg > 0 ? fmaf(a.w, v[4 * q + 3], t[4 * q + 3]) : a.w * v[4 * q + 3];
-              }
-              tmem_st32(tmem_base + lane_off + (uint32_t)BN + col + (uint32_t)(c * 32), t);
+            for (int q = 0; q < 8; ++q) {
+              const float4 a = cb[c * 8 + q];
+              tot[c * 32 + 4 * q] = fmaf(a.x, v0[4 * q], tot[c * 32 + 4 * q]);
+              tot[c * 32 + 4 * q + 1] = fmaf(a.y, v0[4 * q + 1], tot[c * 32 + 4 * q + 1]);
+              tot[c * 32 + 4 * q + 2] = fmaf(a.z, v0[4 * q + 2], tot[c * 32 + 4 * q + 2]);
+              tot[c * 32 + 4 * q + 3] = fmaf(a.w, v0[4 * q + 3], tot[c * 32 + 4 * q + 3]);
             }
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            if (c + 2 < 4) tmem_ld32_issue(tmem_base + lane_off + col + (uint32_t)((c + 2) * 32), v0);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float4 a = cb[(c + 1) * 8 + q];
+              tot[(c + 1) * 32 + 4 * q] = fmaf(a.x, v1[4 * q], tot[(c + 1) * 32 + 4 * q]);
+              tot[(c + 1) * 32 + 4 * q + 1] = fmaf(a.y, v1[4 * q + 1], tot[(c + 1) * 32 + 4 * q + 1]);
+              tot[(c + 1) * 32 + 4 * q + 2] = fmaf(a.z, v1[4 * q + 2], tot[(c + 1) * 32 + 4 * q + 2]);
+              tot[(c + 1) * 32 + 4 * q + 3] = fmaf(a.w, v1[4 * q + 3], tot[(c + 1) * 32 + 4 * q + 3]);
+            }
           }
-          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&pempty_bar[h]);      // also after a failed wait: nobody is left waiting on this warp
         }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&pempty_bar[b]);        // also after a failed wait: nobody is left waiting on this warp
       }
-      // One decision for all eight warps (they meet at the named barrier once per group, so none may leave alone):
-      // a wait that gave up anywhere in the CTA has raised the flag.
+      // One decision for all eight warps (none may leave a tile alone: the other warps of its warpgroup wait for it
+      // at the named barrier of the next group): a wait that gave up anywhere in the CTA has raised the flag.
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (*abort_flag) break;
-      // the tile's totals are complete: conv + SiLU on this warp's two page slots
+      // the tile's totals are complete: conv + SiLU on this warpgroup's two page slots
       float cw[4] = {0.f, 0.f, 0.f, 0.f};
       if (ch < p.n_kv) {
         const uint2 wv = *(const uint2*)(p.conv_w + (long long)(p.n_q + ch) * SR_CONV_W);
@@ -519,14 +517,12 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 #pragma unroll
         for (int q = 0; q < 4; ++q) cw[q] = __bfloat162float(w4[q]);
       }
-#pragma unroll 1
-      for (int sl = hw; sl < SLOTS; sl += 2) {
-        const int slot = SLOTS * tt + sl;
-        float v[64], z1, z2, z3;
-        tmem_ld32(tmem_base + lane_off + (uint32_t)(BN + sl * 64), v);
-        tmem_ld32(tmem_base + lane_off + (uint32_t)(BN + sl * 64 + 32), v + 32);
+#pragma unroll
+      for (int sl = 0; sl < 2; ++sl) {
+        const int slot = SLOTS * tt + 2 * wg + sl;
+        float z1, z2, z3;
         load_history(p, false, p.s.slot_first[slot], ch, z1, z2, z3);
-        emit_slot(p, false, ch, ch_local, ct, slot, true, p.s.slot_rows[slot], v, cw, z1, z2, z3);
+        emit_slot(p, false, ch, ch_local, ct, slot, true, p.s.slot_rows[slot], tot + sl * 64, cw, z1, z2, z3);
       }
     }
   }
@@ -849,7 +845,7 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   const long long max_tiles = t_tiles * (a8 ? p.n_ct : p.n_ct + 1);
   int grid = (int)(max_tiles < sm_count ? max_tiles : sm_count);
   if (grid < 1) grid = 1;
-  if (a8) sr_proj_w8a8_kernel<<<grid, NUM_THREADS_SCALED, W8_SMEM_BYTES, stream>>>(map_x, map_w, p);
+  if (a8) sr_proj_w8a8_kernel<<<grid, W8_THREADS, W8_SMEM_BYTES, stream>>>(map_x, map_w, p);
   else if (scaled) sr_proj_fused_kernel<true><<<grid, NUM_THREADS_SCALED, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
   else sr_proj_fused_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
   return cudaGetLastError();
