@@ -272,6 +272,71 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_group(args, wl, dev, rank, world, warmup):
+    """A group workload (Section 4.1: one anchor per group of linear-attention layers): times sr_replay_group_states.
+    A side workload, not the headline configuration: no host-buffer arm and no oracle arm."""
+    import torch
+    from paper_2609_33477_b200 import binding
+    spec = wl.spec
+    rep = binding.Replayer(wl)
+    stream = torch.cuda.current_stream(dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    for _ in range(warmup):
+        rep.replay_group_states(stream=stream)
+    torch.cuda.synchronize(dev)
+    assert rep.group_device_status() == 0
+    launches = rep.last_launch_count()
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = []
+    sampler.start()
+    for i in range(args.steps):
+        flush.fill_(i & 0xFF)
+        e0.record(stream)
+        rep.replay_group_states(stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        times.append(e0.elapsed_time(e1))
+    clocks = sampler.stop()
+    total_ms = max_over_ranks(sum(times), dev)
+    ms = total_ms / args.steps
+    binding.sr_profile_enable(rep.ctx, True)
+    rep.replay_group_states(stream=stream)
+    torch.cuda.synchronize(dev)
+    kernel_ms = {}
+    for k, kind in binding.KERNEL_KINDS.items():
+        t, n = binding.sr_profile_read(rep.ctx, kind)
+        kernel_ms[k] = {"ms": t, "launches": n} if n else None
+    binding.sr_profile_enable(rep.ctx, False)
+    hv = spec.n_v_heads * spec.d_v
+    L = spec.n_layers
+    proj = L * 2.0 * spec.d_model * (spec.conv_channels + 2 * spec.n_v_heads)
+    block = (L - 1) * 4.0 * spec.d_model * hv + sum(6.0 * spec.d_model * f for f in spec.d_ff[:L - 1])
+    rows = wl.total_rows
+    peaks = measured_peaks()
+    gb = kernel_ms.get("group_block")
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": world * rows * L / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": spec.name, "group_layers": L, "d_model": spec.d_model, "heads": spec.n_v_heads,
+                       "d_head": spec.d_k, "d_ff": list(spec.d_ff), "requests": spec.n_requests, "replayed_rows": rows,
+                       "l2": "256 MB flush buffer written between timed steps"},
+            "clocks": clocks, "e2e": None, "gpu_launches": launches * args.steps,
+            "roofline": {"kernel": "all dense products of the group (projections, output gate, output projection, MLP) over "
+                                   "the call time", "bound": "tensor", "achieved": (proj + block) * rows / (ms * 1e-3) / 1e12,
+                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": (proj + block) * rows / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                         "peak_source": f"{peaks['source']} bf16 burst", "traffic": None, "kernel_ms": kernel_ms,
+                         "block_tflops": (block * rows / (gb["ms"] * 1e-3) / 1e12) if gb else None},
+            "cpu_baseline": None}), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -322,6 +387,9 @@ def main():
     warmup = max(args.warmup, 3)
     wl = synth.build_workload(args.config, device=dev, seed=0)
     spec = wl.spec
+    if spec.group:
+        run_group(args, wl, dev, rank, world, warmup)
+        return
     rep = binding.Replayer(wl)
     stream = torch.cuda.current_stream(dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)     # > the 126 MB L2

@@ -28,6 +28,7 @@ struct GemmParams {
   int32_t k_blocks;      // K / 64
   int32_t n;             // output columns (for SWIGLU: hidden width f; the tile holds 128 gate + 128 up columns)
   int32_t n_tiles;
+  int32_t n_block;       // column tiles per weight block of the tile order
   __nv_bfloat16* c;      // [rows][ldc]
   int64_t ldc;
   const __nv_bfloat16* residual;   // EPI_ADD: [rows][ldr]
@@ -72,11 +73,17 @@ sr_rows_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  // tile -> (row tile, column tile): column-fastest, so CTAs running side by side share the rows in L2 and the
-  // weights (a few MB for the widths of a replay batch) stay resident
+  // tile -> (row tile, column tile).  The column tiles are cut into blocks of n_block tiles whose weights (about
+  // 24 MB) stay in L2 while every row tile streams past them, column-fastest inside the block: weights come from
+  // HBM once, rows once per block.  (Column-fastest over the whole width re-read a 105 MB weight matrix once per
+  // two row tiles: 1.6 GB of HBM reads for 0.13 GB of operands on 4096 rows.)
   auto tile_coords = [&](long long tile, int& mt, int& nt) {
-    mt = (int)(tile / p.n_tiles);
-    nt = (int)(tile % p.n_tiles);
+    const long long per_block = (long long)m_tiles * p.n_block;
+    const int blk = (int)(tile / per_block);
+    const int r = (int)(tile - blk * per_block);
+    const int nbt = min(p.n_block, p.n_tiles - blk * p.n_block);
+    mt = r / nbt;
+    nt = blk * p.n_block + r % nbt;
   };
 
   if (warp == 0) {
@@ -296,6 +303,13 @@ cudaError_t sr_launch_rows_gemm(const SrSched& s, int kind, const __nv_bfloat16*
   p.n = n;
   const int ncol = kind == EPI_SWIGLU ? GN / 2 : GN;
   p.n_tiles = (n + ncol - 1) / ncol;
+  {
+    const long long tile_bytes = (long long)GN * k * 2;       // weight rows one tile reads (both halves of a SwiGLU tile)
+    long long nb = (24ll << 20) / tile_bytes;
+    if (nb < 1) nb = 1;
+    const long long blocks = (p.n_tiles + nb - 1) / nb;       // equal blocks
+    p.n_block = (int32_t)((p.n_tiles + blocks - 1) / blocks);
+  }
   p.c = c;
   p.ldc = ldc;
   p.residual = residual;
