@@ -52,6 +52,13 @@ def _close_rows(got_bits, ref_bits, what, hops, aggregate=True):
     return float((got_bits == ref_bits).mean())
 
 
+def _strict_conv(tail_gpu, tail_ref):
+    """The single-layer rule: one bf16 step at most (entries next to zero: 1e-5 absolute), nearly all identical."""
+    dist = U.bf16_ulp_distance(tail_gpu, tail_ref)
+    a, b = orc.bf16_bits_to_f64(tail_gpu), orc.bf16_bits_to_f64(tail_ref)
+    assert ((dist <= 1) | (np.abs(a - b) <= 1e-5)).all() and (dist > 0).mean() <= 0.02
+
+
 def _oracle_group(wl, i):
     s = wl.spec
     R = int(wl.replay_lens[i].item())
@@ -83,9 +90,7 @@ def test_group_states_and_handed_rows_match_the_oracle(name):
             assert err <= tol, f"{name} request {i} layer {l}: rel Frobenius {err:.3e} > {tol}"
             tail_gpu = _bits(rep.out_conv[i, l])
             if l == 0:
-                dist = U.bf16_ulp_distance(tail_gpu, tail_ref)
-                a, b = orc.bf16_bits_to_f64(tail_gpu), orc.bf16_bits_to_f64(tail_ref)
-                assert ((dist <= 1) | (np.abs(a - b) <= 1e-5)).all() and (dist > 0).mean() <= 0.02
+                _strict_conv(tail_gpu, tail_ref)
             else:
                 _close_rows(tail_gpu.T, tail_ref.T, f"{name} request {i} layer {l} conv state", hops=l, aggregate=False)
         for j, ref_bits in enumerate(handed):
@@ -109,3 +114,27 @@ def test_a_group_of_one_layer_and_the_prefix_of_a_longer_group_agree():
     assert torch.equal(rep.out_ssm[:, :2], full_ssm[:, :2]) and torch.equal(rep.out_conv[:, :2], full_conv[:, :2])
     assert not rep.out_ssm[:, 2].any()                      # the third layer was not touched
     assert rep.last_launch_count() > 0
+
+
+def test_group_at_the_benchmarked_size_matches_the_oracle_on_sampled_requests():
+    """`group3_4b` as `bench.py --config group3_4b` runs it (three layers of the 4B geometry with MLPs, eight 512-row
+    requests, 4096 packed rows): two requests are replayed by the oracle and every layer of the group is compared."""
+    wl = synth.build_workload("group3_4b", device="cuda")
+    rep = binding.Replayer(wl)
+    st, rows = rep.replay_group_states(debug_rows=True)
+    torch.cuda.synchronize()
+    assert st == 0 and rep.group_device_status() == 0
+    lens = wl.replay_lens.cpu().tolist()
+    for i in (0, 5):
+        res, handed = _oracle_group(wl, i)
+        slot0 = sum(-(-r // 64) for r in lens[:i])
+        for l, (S_ref, tail_ref) in enumerate(res):
+            err = U.rel_frob_per_head(rep.out_ssm[i, l].cpu().numpy(), S_ref)
+            assert err <= U.REL_FROB_TOL + 1e-2 * l, f"request {i} layer {l}: rel Frobenius {err:.3e}"
+            tail_gpu = _bits(rep.out_conv[i, l])
+            if l == 0:
+                _strict_conv(tail_gpu, tail_ref)
+            else:
+                _close_rows(tail_gpu.T, tail_ref.T, f"request {i} layer {l} conv state", hops=l, aggregate=False)
+        for j, ref_bits in enumerate(handed):
+            _close_rows(_bits(rows[j, slot0 * 64: slot0 * 64 + lens[i]]), ref_bits, f"request {i} rows after layer {j}", hops=j + 1)
