@@ -62,6 +62,7 @@ cudaError_t sr_current_device_sms(int* sms);
 // Scratch layout inside the caller's workspace (all offsets in bytes, 256-aligned).
 struct sr_ctx;
 size_t sr_scan_split_bytes(const sr_ctx* ctx, int64_t max_slots);
+size_t sr_conv_tail_part_bytes(const sr_ctx* ctx);
 
 struct SrWorkspace {
   size_t off_header;     // uint32 status, int32 n_slots, int32 total_rows
@@ -83,6 +84,7 @@ struct SrWorkspace {
   size_t off_x16;        // fp16 staging: half [max_slots][64][d_model] anchors of the current layer, slot order;
                          // W8A8: uint8 [max_slots][64][d_model] activation codes
   size_t off_sx;         // W8A8: float [max_slots][d_model / 128][64] activation scales
+  size_t off_qpart;      // float [4][256][channels] partial sums of the conv-state kernel's k quarters (small batches)
   size_t lane_bytes;     // size of one lane's block of hand-over buffers (off_kv16 .. end)
   int lanes;             // lane blocks in `total`
   size_t total;
@@ -124,6 +126,7 @@ static inline SrWorkspace sr_workspace_layout(const sr_ctx* ctx, int32_t n_reque
                                                                                      (size_t)ctx->desc.d_model : 0));
   w.off_sx = at;        at = sr_align256(at + (ctx->w8a8 ? sizeof(float) * (size_t)w.max_slots * SR_PAGE_ROWS *
                                                                (size_t)(ctx->desc.d_model / 128) : 0));
+  w.off_qpart = at;     at = sr_align256(at + ((int64_t)n_requests * (SR_CONV_W - 1) <= 256 ? sr_conv_tail_part_bytes(ctx) : 0));
   at = (at + 1023) & ~size_t(1023);
   w.lane_bytes = at - lane0;
   w.lanes = lanes < 1 ? 1 : lanes;
@@ -229,6 +232,7 @@ struct SrFused {
   // group replay only: what the state chain leaves for the output kernel, per (slot, value head)
   __half* dump_s;    // [slot][H_v][d_k][d_v] fp16: the state entering the chunk (not written for a request's first chunk)
   __half* dump_u;    // [slot][H_v][d_v][64] fp16: the chunk's pseudo-values U^T, before the row factors
+  float* qpart;      // conv state of small batches: partial sums of the batched kernel's k quarters, or null
 };
 
 struct SrPoolView {

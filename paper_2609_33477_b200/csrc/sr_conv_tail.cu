@@ -122,6 +122,8 @@ sr_conv_tail_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_mo
 constexpr int QT = 64;            // tile rows, tile channels and k chunk
 constexpr int QLD = QT + 8;       // shared-memory pitch (bf16)
 constexpr int QNS = 4;            // chunks in flight: the k loop is serial, so its speed is latency / depth
+constexpr int QR = 4;             // quarters the k range is always summed in (see the kernel)
+constexpr int SPLIT_MAX_ROWS = 256;   // tail rows (3 per request) up to which every quarter gets its own CTA
 
 template <bool FP8, bool A8>
 constexpr int conv_gemm_smem() {
@@ -136,7 +138,8 @@ __global__ void __launch_bounds__(128)
 sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_model, int32_t conv_ch,
                          const void* __restrict__ w_rows, const float* __restrict__ w_scale,
                          const uint8_t* __restrict__ x8, const float* __restrict__ sx,
-                         const __nv_bfloat16* __restrict__ hist, char* __restrict__ out_layer, int64_t slot_stride) {
+                         const __nv_bfloat16* __restrict__ hist, char* __restrict__ out_layer, int64_t slot_stride,
+                         float* __restrict__ part, int32_t part_rows, int32_t part_ch) {
   // Shared memory: a ring of QNS stages per operand.  A 16-bit operand is copied straight into its padded tile
   // (cp.async, 16 bytes); an 8-bit operand lands as raw bytes (cp.async, 8 bytes) and the thread that fetched them
   // decodes them into one of two bf16 tiles just before the chunk is used.
@@ -173,8 +176,8 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
     // bf16: 16 bytes = 8 weights per thread and row; e4m3: 8 bytes = 8 codes
     wrow[q] = (const char*)w_rows + ((int64_t)(c0 + m) * d_model + seg * 8) * (FP8 ? 1 : 2);
   }
-  auto load = [&](int kc) {            // chunk kc -> ring stage kc % QNS
-    const int st = kc % QNS;
+  auto load = [&](int kc, int ring) {  // chunk kc -> ring stage ring % QNS
+    const int st = ring % QNS;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int m = (tid >> 3) + 16 * q;
@@ -228,48 +231,88 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
       for (int c = 0; c < 4; ++c) { acc[rb][n][c] = 0.f; total[rb][n][c] = 0.f; }
   const int nk = d_model / QT;
   const float* scale_row = FP8 ? w_scale + (int64_t)(c0 / 128) * (d_model / 128) : nullptr;
-  for (int kc = 0; kc < QNS - 1; ++kc) {       // fill the ring; one commit group per chunk, empty ones past the end
-    if (kc < nk) load(kc);
-    asm volatile("cp.async.commit_group;" ::: "memory");
-  }
-  for (int kc = 0; kc < nk; ++kc) {
-    asm volatile("cp.async.wait_group %0;" ::"n"(QNS - 2) : "memory");      // this thread's part of chunk kc has landed
-    const __half* xt = A8 ? Xt + (kc & 1) * (QT * QLD) : Xt + (kc % QNS) * (QT * QLD);
-    const __half* wt = FP8 ? Wt + (kc & 1) * (QT * QLD) : Wt + (kc % QNS) * (QT * QLD);
-    if (A8) decode_own(Xraw + (kc % QNS) * RAW_B, (__half*)xt);
-    if (FP8) decode_own(Wraw + (kc % QNS) * RAW_B, (__half*)wt);
-    __syncthreads();                  // chunk kc is complete for everyone; everyone is done with chunk kc - 1
-    if (kc + QNS - 1 < nk) load(kc + QNS - 1);                             // into the stage chunk kc - 1 used
-    asm volatile("cp.async.commit_group;" ::: "memory");
+  // The sum over k is ALWAYS formed as ((r_0 + r_1) + r_2) + r_3, r_z the sum over the z-th quarter of the chunks
+  // (quarters of the 128-deep groups for block-scaled weights): a small batch gives every quarter its own CTA
+  // (gridDim.z = QR, partial sums to `part`, added up by the finishing kernel), a large one walks the quarters in
+  // one CTA -- the same numbers added in the same order, so a request's conv state does not depend on the batch it
+  // arrives in.
+  float fin[4][2][4];
 #pragma unroll
-    for (int ks = 0; ks < QT / 16; ++ks) {
-      uint32_t bf[4];
-      ldsm4(bf, bn_addr(wt, QLD, warp * 16, ks * 16, l));
+  for (int rb = 0; rb < 4; ++rb)
 #pragma unroll
-      for (int rb = 0; rb < 4; ++rb) {
-        if (rb < n_rb) {
-          uint32_t a[4];
-          ldsm4(a, a_addr(xt, QLD, rb * 16, ks * 16, l));
-          mma16816_bf16(acc[rb][0], a, bf[0], bf[1]);
-          mma16816_bf16(acc[rb][1], a, bf[2], bf[3]);
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) fin[rb][n][c] = 0.f;
+  const int z0 = part ? (int)blockIdx.z : 0, z1 = part ? z0 + 1 : QR;
+  for (int z = z0; z < z1; ++z) {
+    const int kb = FP8 ? 2 * ((z * (nk / 2)) / QR) : (z * nk) / QR;
+    const int ke = FP8 ? 2 * (((z + 1) * (nk / 2)) / QR) : ((z + 1) * nk) / QR;
+    for (int kc = kb; kc < kb + QNS - 1; ++kc) {       // fill the ring; one commit group per chunk, empty ones past the end
+      if (kc < ke) load(kc, kc - kb);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    for (int kc = kb; kc < ke; ++kc) {
+      const int ring = kc - kb;
+      asm volatile("cp.async.wait_group %0;" ::"n"(QNS - 2) : "memory");      // this thread's part of chunk kc has landed
+      const __half* xt = A8 ? Xt + (ring & 1) * (QT * QLD) : Xt + (ring % QNS) * (QT * QLD);
+      const __half* wt = FP8 ? Wt + (ring & 1) * (QT * QLD) : Wt + (ring % QNS) * (QT * QLD);
+      if (A8) decode_own(Xraw + (ring % QNS) * RAW_B, (__half*)xt);
+      if (FP8) decode_own(Wraw + (ring % QNS) * RAW_B, (__half*)wt);
+      __syncthreads();                  // chunk kc is complete for everyone; everyone is done with chunk kc - 1
+      if (kc + QNS - 1 < ke) load(kc + QNS - 1, ring + QNS - 1);             // into the stage chunk kc - 1 used
+      asm volatile("cp.async.commit_group;" ::: "memory");
+#pragma unroll
+      for (int ks = 0; ks < QT / 16; ++ks) {
+        uint32_t bf[4];
+        ldsm4(bf, bn_addr(wt, QLD, warp * 16, ks * 16, l));
+#pragma unroll
+        for (int rb = 0; rb < 4; ++rb) {
+          if (rb < n_rb) {
+            uint32_t a[4];
+            ldsm4(a, a_addr(xt, QLD, rb * 16, ks * 16, l));
+            mma16816_bf16(acc[rb][0], a, bf[0], bf[1]);
+            mma16816_bf16(acc[rb][1], a, bf[2], bf[3]);
+          }
+        }
+      }
+      if (FP8 && (kc & 1)) {         // a 128-deep k group is complete: it shares one block scale
+        const float sc = __ldg(scale_row + (kc >> 1));
+#pragma unroll
+        for (int rb = 0; rb < 4; ++rb) {
+          if (rb < n_rb) {
+            const float s0 = A8 ? sc * __ldg(sxrow[rb][0] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
+            const float s1 = A8 ? sc * __ldg(sxrow[rb][1] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+              for (int c = 0; c < 4; ++c) { total[rb][n][c] = fmaf(c < 2 ? s0 : s1, acc[rb][n][c], total[rb][n][c]); acc[rb][n][c] = 0.f; }
+          }
         }
       }
     }
-    if (FP8 && (kc & 1)) {         // a 128-deep k group is complete: it shares one block scale
-      const float sc = __ldg(scale_row + (kc >> 1));
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();                    // the ring is idle before the next quarter refills it
+    // this quarter's sum: into the running total, or out to the partial-sum buffer
 #pragma unroll
-      for (int rb = 0; rb < 4; ++rb) {
-        if (rb < n_rb) {
-          const float s0 = A8 ? sc * __ldg(sxrow[rb][0] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
-          const float s1 = A8 ? sc * __ldg(sxrow[rb][1] + (int64_t)(kc >> 1) * SR_PAGE_ROWS) : sc;
+    for (int rb = 0; rb < 4; ++rb)
 #pragma unroll
-          for (int n = 0; n < 2; ++n)
+      for (int n = 0; n < 2; ++n) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) { total[rb][n][c] = fmaf(c < 2 ? s0 : s1, acc[rb][n][c], total[rb][n][c]); acc[rb][n][c] = 0.f; }
+        for (int c = 0; c < 4; ++c) {
+          const float r = FP8 ? total[rb][n][c] : acc[rb][n][c];
+          fin[rb][n][c] += r;
+          acc[rb][n][c] = 0.f;
+          total[rb][n][c] = 0.f;
+        }
+        if (part && rb < n_rb) {
+          const int ch = c0 + warp * 16 + n * 8 + 2 * t4;
+          float* dstp = part + ((int64_t)z * part_rows + r0 + rb * 16 + g8) * part_ch + ch;
+          *(float2*)dstp = make_float2(fin[rb][n][0], fin[rb][n][1]);
+          *(float2*)(dstp + (int64_t)8 * part_ch) = make_float2(fin[rb][n][2], fin[rb][n][3]);
         }
       }
-    }
   }
+  if (part) return;                     // the finishing kernel adds the quarters up and writes the state
 #pragma unroll
   for (int rb = 0; rb < 4; ++rb) {
 #pragma unroll
@@ -285,7 +328,7 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
 #pragma unroll
       for (int n = 0; n < 2; ++n) {
         const int c = c0 + warp * 16 + n * 8 + 2 * t4;
-        const float v0 = FP8 ? total[rb][n][2 * hr] : acc[rb][n][2 * hr], v1 = FP8 ? total[rb][n][2 * hr + 1] : acc[rb][n][2 * hr + 1];
+        const float v0 = fin[rb][n][2 * hr], v1 = fin[rb][n][2 * hr + 1];
         __nv_bfloat16 o0 = __float2bfloat16_rn(t >= 0 ? v0 : 0.f), o1 = __float2bfloat16_rn(t >= 0 ? v1 : 0.f);
         if (old) {
           o0 = old[(int64_t)c * (SR_CONV_W - 1)];
@@ -298,17 +341,20 @@ sr_conv_tail_gemm_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t
   }
 }
 
-// k and v channels from the rows the fused projection kept: one thread per (request, channel), so the reads of a
-// row are contiguous across the warp and a thread writes its channel's w-1 entries side by side
+// k and v channels from the rows the fused projection kept, and the channels whose k quarters were summed by separate
+// CTAs (`part`: [quarter][tail row][channel], channels 0 .. part_ch - 1): one thread per (request, channel), so the
+// reads of a row are contiguous across the warp and a thread writes its channel's w-1 entries side by side
 __global__ void __launch_bounds__(256)
-sr_conv_tail_kv_kernel(SrSched s, int32_t n_q, int32_t conv_ch, const float* __restrict__ zraw, int32_t n_kv,
-                       const __nv_bfloat16* __restrict__ hist, char* __restrict__ out_layer, int64_t slot_stride) {
+sr_conv_tail_kv_kernel(SrSched s, int32_t c_begin, int32_t n_q, int32_t conv_ch, const float* __restrict__ zraw, int32_t n_kv,
+                       const __nv_bfloat16* __restrict__ hist, char* __restrict__ out_layer, int64_t slot_stride,
+                       const float* __restrict__ part, int32_t part_rows, int32_t part_ch) {
   const int i = blockIdx.y;
   const int out_slot = s.req_out[i];
   if (out_slot < 0) return;
-  const int ckv = blockIdx.x * blockDim.x + threadIdx.x;
-  if (ckv >= n_kv) return;
-  const int c = n_q + ckv;
+  const int c = c_begin + blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= conv_ch) return;
+  const bool from_part = part && c < part_ch;
+  if (!from_part && c < n_q) return;              // written by the batched kernel itself
   const int R = s.req_rows[i], slot0 = s.req_slot0[i];
   if (!sr_check_out(s, out_slot) || (R > 0 && !sr_check_slot(s, slot0 + (R - 1) / SR_PAGE_ROWS))) return;
   __nv_bfloat16* dst = (__nv_bfloat16*)(out_layer + (int64_t)out_slot * slot_stride) + (int64_t)c * (SR_CONV_W - 1);
@@ -317,9 +363,17 @@ sr_conv_tail_kv_kernel(SrSched s, int32_t n_q, int32_t conv_ch, const float* __r
     const int t = R - (SR_CONV_W - 1) + j;
     __nv_bfloat16 o = __float2bfloat16_rn(0.f);
     if (t >= 0) {
-      const int slot = slot0 + t / SR_PAGE_ROWS, rho = t % SR_PAGE_ROWS;
-      const int idx = 3 + rho - max(s.slot_rows[slot] - 3, 0);
-      o = __float2bfloat16_rn(zraw[((int64_t)slot * 6 + idx) * n_kv + ckv]);
+      if (from_part) {
+        const int64_t gr = (int64_t)i * (SR_CONV_W - 1) + j;
+        float v = 0.f;
+#pragma unroll
+        for (int z = 0; z < QR; ++z) v += part[((int64_t)z * part_rows + gr) * part_ch + c];
+        o = __float2bfloat16_rn(v);
+      } else {
+        const int slot = slot0 + t / SR_PAGE_ROWS, rho = t % SR_PAGE_ROWS;
+        const int idx = 3 + rho - max(s.slot_rows[slot] - 3, 0);
+        o = __float2bfloat16_rn(zraw[((int64_t)slot * 6 + idx) * n_kv + (c - n_q)]);
+      }
     } else if (hist) {
       o = hist[((int64_t)i * conv_ch + c) * (SR_CONV_W - 1) + (SR_CONV_W - 1 + t)];
     }
@@ -351,9 +405,19 @@ static bool conv_tail_gemm_fits(const sr_ctx* ctx, int n_requests) {
          !(ctx->debug_flags & SR_DEBUG_DOT_CONV_STATE);
 }
 
+static bool conv_tail_split(const sr_ctx* ctx, int n_requests) {
+  return conv_tail_gemm_fits(ctx, n_requests) && n_requests * (SR_CONV_W - 1) <= SPLIT_MAX_ROWS;
+}
+
 int sr_conv_tail_launches(const sr_ctx* ctx, int n_requests) {
   if (!conv_tail_gemm_fits(ctx, n_requests)) return 1;
-  return ctx->desc.weight_format == SR_W_E4M3_BLOCK128 ? 1 : 2;
+  return (ctx->desc.weight_format == SR_W_E4M3_BLOCK128 && !conv_tail_split(ctx, n_requests)) ? 1 : 2;
+}
+
+// bytes of the partial-sum buffer a lane needs (small batches: the k quarters are summed by separate CTAs)
+size_t sr_conv_tail_part_bytes(const sr_ctx* ctx) {
+  const size_t ch = ctx->desc.weight_format == SR_W_E4M3_BLOCK128 ? ctx->conv_ch : ctx->n_k;
+  return (size_t)QR * SPLIT_MAX_ROWS * ch * sizeof(float);
 }
 
 cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoolView& pool, int32_t pool_layer,
@@ -375,40 +439,45 @@ cudaError_t sr_launch_conv_tail(const sr_ctx* ctx, const SrSched& s, const SrPoo
     return e;
   });
   if (once != cudaSuccess) return once;
-  if (ctx->desc.weight_format == SR_W_E4M3_BLOCK128) {
-    // every channel from codes and scales in fp32: the conv state never sees a rounded weight
-    if (conv_tail_gemm_fits(ctx, s.n_requests)) {
-      dim3 g((unsigned)(ctx->conv_ch / QT), (unsigned)((tail_rows + QT - 1) / QT));
-      if (ctx->w8a8)
-        sr_conv_tail_gemm_kernel<true, true><<<g, 128, conv_gemm_smem<true, true>(), stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
-                                                                    w.w_qkv_scale, fused.x8, fused.sx, hist, out_conv_layer,
-                                                                    slot_stride);
-      else
-        sr_conv_tail_gemm_kernel<true, false><<<g, 128, conv_gemm_smem<true, false>(), stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
-                                                                     w.w_qkv_scale, nullptr, nullptr, hist, out_conv_layer,
-                                                                     slot_stride);
-      return cudaGetLastError();
-    }
-    dim3 grid((unsigned)((ctx->conv_ch + 7) / 8), (unsigned)s.n_requests);
-    sr_conv_tail_kernel<true><<<grid, 256, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, 0,
-                                                        ctx->conv_ch, w.w_qkv, w.w_qkv_scale, zraw, n_kv, hist,
-                                                        out_conv_layer, slot_stride);
-    return cudaGetLastError();
-  }
-  // bf16 weights: the q channels as one batched GEMM (or by dot products), the k and v channels copied from the
-  // raw rows the projection kept
+  const bool fp8 = ctx->desc.weight_format == SR_W_E4M3_BLOCK128;
   const int n_q = ctx->n_k;
   if (conv_tail_gemm_fits(ctx, s.n_requests)) {
-    dim3 gq((unsigned)(n_q / QT), (unsigned)((tail_rows + QT - 1) / QT));
-    sr_conv_tail_gemm_kernel<false, false><<<gq, 128, conv_gemm_smem<false, false>(), stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv,
-                                                                    nullptr, nullptr, nullptr, hist, out_conv_layer, slot_stride);
-    dim3 gkv((unsigned)((n_kv + 255) / 256), (unsigned)s.n_requests);
-    sr_conv_tail_kv_kernel<<<gkv, 256, 0, stream>>>(s, n_q, ctx->conv_ch, zraw, n_kv, hist, out_conv_layer, slot_stride);
+    // the batched kernel: the q channels (bf16 weights; k and v rows come from the raw rows the projection kept), or
+    // every channel from codes and scales in fp32 (block-scaled weights: the conv state never sees a rounded weight)
+    const int gemm_ch = fp8 ? ctx->conv_ch : n_q;
+    const bool split = conv_tail_split(ctx, s.n_requests) && fused.qpart != nullptr;
+    const int row_tiles = (tail_rows + QT - 1) / QT;
+    float* part = split ? fused.qpart : nullptr;
+    const int part_rows = row_tiles * QT;
+    dim3 g((unsigned)(gemm_ch / QT), (unsigned)row_tiles, split ? QR : 1);
+    if (!fp8)
+      sr_conv_tail_gemm_kernel<false, false><<<g, 128, conv_gemm_smem<false, false>(), stream>>>(
+          s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv, nullptr, nullptr, nullptr, hist, out_conv_layer, slot_stride,
+          part, part_rows, gemm_ch);
+    else if (ctx->w8a8)
+      sr_conv_tail_gemm_kernel<true, true><<<g, 128, conv_gemm_smem<true, true>(), stream>>>(
+          s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv, w.w_qkv_scale, fused.x8, fused.sx, hist, out_conv_layer,
+          slot_stride, part, part_rows, gemm_ch);
+    else
+      sr_conv_tail_gemm_kernel<true, false><<<g, 128, conv_gemm_smem<true, false>(), stream>>>(
+          s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, w.w_qkv, w.w_qkv_scale, nullptr, nullptr, hist, out_conv_layer,
+          slot_stride, part, part_rows, gemm_ch);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || (fp8 && !split)) return e;
+    // the k | v copy (bf16 weights) and, for a split sum, the channels whose quarters are added up here
+    const int c_begin = split ? 0 : n_q;
+    dim3 gkv((unsigned)((ctx->conv_ch - c_begin + 255) / 256), (unsigned)s.n_requests);
+    sr_conv_tail_kv_kernel<<<gkv, 256, 0, stream>>>(s, c_begin, fp8 ? ctx->conv_ch : n_q, ctx->conv_ch, zraw, n_kv, hist, out_conv_layer,
+                                                    slot_stride, part, part_rows, gemm_ch);
     return cudaGetLastError();
   }
   dim3 grid((unsigned)((ctx->conv_ch + 7) / 8), (unsigned)s.n_requests);
-  sr_conv_tail_kernel<false><<<grid, 256, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, n_q, 0, ctx->conv_ch,
-                                                       w.w_qkv, nullptr, zraw, n_kv, hist, out_conv_layer, slot_stride);
+  if (fp8)
+    sr_conv_tail_kernel<true><<<grid, 256, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, ctx->conv_ch, 0, ctx->conv_ch, w.w_qkv,
+                                                        w.w_qkv_scale, zraw, n_kv, hist, out_conv_layer, slot_stride);
+  else
+    sr_conv_tail_kernel<false><<<grid, 256, 0, stream>>>(s, pool, pool_layer, ctx->desc.d_model, n_q, 0, ctx->conv_ch, w.w_qkv, nullptr,
+                                                         zraw, n_kv, hist, out_conv_layer, slot_stride);
   return cudaGetLastError();
 }
 
@@ -416,7 +485,8 @@ cudaError_t sr_launch_conv_tail_from_raw(const sr_ctx* ctx, const SrSched& s, co
                                          int64_t slot_stride, cudaStream_t stream) {
   // every conv channel was projected for every row: the last rows are all in zraw (n_q = 0, n_kv = C)
   dim3 g((unsigned)((ctx->conv_ch + 255) / 256), (unsigned)s.n_requests);
-  sr_conv_tail_kv_kernel<<<g, 256, 0, stream>>>(s, 0, ctx->conv_ch, fused.zraw, ctx->conv_ch, nullptr, out_conv_layer, slot_stride);
+  sr_conv_tail_kv_kernel<<<g, 256, 0, stream>>>(s, 0, 0, ctx->conv_ch, fused.zraw, ctx->conv_ch, nullptr, out_conv_layer, slot_stride, nullptr,
+                                                0, 0);
   return cudaGetLastError();
 }
 

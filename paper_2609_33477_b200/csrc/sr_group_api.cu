@@ -159,6 +159,7 @@ extern "C" int sr_replay_group_states(sr_ctx* ctx, const sr_anchor_pool* pool, c
   fused.v_ch0 = 2 * ctx->n_k;
   fused.dump_s = (__half*)(ws + lay.off_dump_s);
   fused.dump_u = (__half*)(ws + lay.off_dump_u);
+  fused.qpart = nullptr;
   void* split = ws + lay.off_split;
   __nv_bfloat16* x = (__nv_bfloat16*)(ws + lay.off_x);
   __nv_bfloat16* r_cur = (__nv_bfloat16*)(ws + lay.off_r0);

@@ -486,3 +486,31 @@ def test_call_is_graph_capturable_with_device_side_boundaries():
             if wl.layer_mask[l]:
                 assert torch.equal(got_ssm[:, l], rep.out_ssm[:, l]) and torch.equal(got_conv[:, l], rep.out_conv[:, l])
     U.check_request_layer(rep, wl, 5, 0)
+
+
+@pytest.mark.parametrize("name", ["many_requests", "fp8_many"])
+def test_a_request_gets_the_same_bits_alone_and_in_a_large_batch(name):
+    """The conv-state kernel gives every quarter of the k range its own CTA on small batches and walks the quarters in
+    one CTA on large ones; the sums are formed in the same order, so both states of a request are bit-identical
+    whatever batch it arrives in (a comparison of the CUDA path with itself; both batch sizes are compared with the
+    oracle elsewhere)."""
+    import dataclasses
+    if name == "fp8_many":
+        spec = dataclasses.replace(synth.SPECS["many_requests"], name="fp8_many", n_requests=120, weight_format="e4m3_block128")
+    else:
+        spec = synth.SPECS[name]
+    wl = synth.build_workload(spec, device="cuda")
+    rep = B.Replayer(wl)
+    rep.replay_states()
+    torch.cuda.synchronize()
+    assert rep.device_status() == 0
+    lens = wl.replay_lens.cpu().tolist()
+    picks = [i for i, r in enumerate(lens) if r > 0][:2] + [max(range(len(lens)), key=lambda i: lens[i])]
+    for i in picks:
+        n_pg = max(1, -(-lens[i] // 64))
+        one = dataclasses.replace(wl, page_table=wl.page_table[i:i + 1, :n_pg].contiguous(), replay_lens=wl.replay_lens[i:i + 1].clone())
+        rep1 = B.Replayer(one)
+        rep1.replay_states()
+        torch.cuda.synchronize()
+        assert torch.equal(rep1.out_conv[0], rep.out_conv[i]) and torch.equal(rep1.out_ssm[0], rep.out_ssm[i])
+        rep1.close()
