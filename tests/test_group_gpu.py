@@ -138,3 +138,44 @@ def test_group_at_the_benchmarked_size_matches_the_oracle_on_sampled_requests():
                 _close_rows(tail_gpu.T, tail_ref.T, f"request {i} layer {l} conv state", hops=l, aggregate=False)
         for j, ref_bits in enumerate(handed):
             _close_rows(_bits(rows[j, slot0 * 64: slot0 * 64 + lens[i]]), ref_bits, f"request {i} rows after layer {j}", hops=j + 1)
+
+
+def _draw_group(seed):
+    r = np.random.RandomState(2000 + seed)
+    d_k = d_v = int(r.choice([64, 128]))
+    h_k = int(r.randint(1, 4))
+    h_v = h_k * int(r.randint(1, 4))
+    n_layers = int(r.randint(2, 4))
+    n_req = int(r.randint(1, 5))
+    lens = tuple(int(x) for x in r.choice([0, 1, 3, 63, 64, 65, 129, 200, 257], size=n_req))
+    d_ff = tuple(int(64 * r.randint(0, 9)) for _ in range(n_layers))
+    return synth.WorkloadSpec(name=f"random_group_{seed}", n_layers=n_layers, d_model=int(64 * r.randint(2, 11)), n_k_heads=h_k,
+                              n_v_heads=h_v, d_k=d_k, d_v=d_v, n_requests=n_req, replay=("list", lens), group=True, d_ff=d_ff,
+                              paging=["shuffled", "identity"][r.randint(2)])
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_groups_match_the_oracle(seed):
+    """Seeded random widths, head counts, group sizes, MLP widths and ragged batches, same comparison as above."""
+    spec = _draw_group(seed)
+    wl = synth.build_workload(spec, device="cuda", seed=seed)
+    rep = binding.Replayer(wl)
+    st, rows = rep.replay_group_states(debug_rows=True)
+    torch.cuda.synchronize()
+    assert st == 0 and rep.group_device_status() == 0
+    slot0 = 0
+    for i, R in enumerate(wl.replay_lens.cpu().tolist()):
+        res, handed = _oracle_group(wl, i)
+        for l, (S_ref, tail_ref) in enumerate(res):
+            S_gpu = rep.out_ssm[i, l].cpu().numpy()
+            assert np.all(np.isfinite(S_gpu))
+            err = U.rel_frob_per_head(S_gpu, S_ref)
+            assert err <= U.REL_FROB_TOL + 1e-2 * l, f"{spec} request {i} layer {l}: rel Frobenius {err:.3e}"
+            tail_gpu = _bits(rep.out_conv[i, l])
+            if l == 0:
+                _strict_conv(tail_gpu, tail_ref)
+            else:
+                _close_rows(tail_gpu.T, tail_ref.T, f"request {i} layer {l} conv state", hops=l, aggregate=False)
+        for j, ref_bits in enumerate(handed):
+            _close_rows(_bits(rows[j, slot0 * 64: slot0 * 64 + R]), ref_bits, f"request {i} rows after layer {j}", hops=j + 1)
+        slot0 += -(-R // 64)
