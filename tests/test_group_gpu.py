@@ -179,3 +179,22 @@ def test_random_groups_match_the_oracle(seed):
         for j, ref_bits in enumerate(handed):
             _close_rows(_bits(rows[j, slot0 * 64: slot0 * 64 + R]), ref_bits, f"request {i} rows after layer {j}", hops=j + 1)
         slot0 += -(-R // 64)
+
+
+def test_the_group_call_can_be_captured_in_a_cuda_graph():
+    """No host synchronisation, no allocation: one captured graph replays the whole group call bit for bit."""
+    wl = synth.build_workload("group_small", device="cuda")
+    rep = binding.Replayer(wl)
+    rep.replay_group_states()                        # one-time kernel attributes and the workspace, outside the capture
+    torch.cuda.synchronize()
+    ref_ssm, ref_conv = rep.out_ssm.clone(), rep.out_conv.clone()
+    rep.out_ssm.zero_()
+    rep.out_conv.zero_()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        rep.replay_group_states(stream=torch.cuda.current_stream())
+    graph.replay()
+    torch.cuda.synchronize()
+    assert rep.group_device_status() == 0
+    assert torch.equal(rep.out_ssm, ref_ssm) and torch.equal(rep.out_conv, ref_conv)
