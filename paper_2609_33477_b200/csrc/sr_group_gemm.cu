@@ -209,19 +209,20 @@ sr_rows_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   }
 }
 
-// x[slot][row][:] = bf16( r * rsqrt(mean(r^2) + eps) * w ), one warp per row.  The rows come from the anchor pool
+// x[slot][row][:] = bf16( r * rsqrt(mean(r^2) + eps) * w ), one warp per row, eight rows per CTA.  The rows come from the anchor pool
 // through the slot table (the group's first layer) or from a packed row buffer (the later ones); rows past a
 // window's end are written as zeros, whatever the source holds there.
 __global__ void __launch_bounds__(256)
 sr_rmsnorm_rows_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, const __nv_bfloat16* __restrict__ rows_in,
                        const __nv_bfloat16* __restrict__ w, float eps, int32_t d_model, __nv_bfloat16* __restrict__ out,
                        __nv_bfloat16* __restrict__ copy_out) {
-  const int slot = blockIdx.x;
+  const int slot = blockIdx.x >> 3;                       // eight CTAs per page slot, a warp per row
   if (slot >= (((int)s.status[1] + 3) & ~3)) return;
   const int vr = s.slot_rows[slot];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nvec = d_model / 8;
-  for (int r = warp; r < SR_PAGE_ROWS; r += 8) {
+  {
+    const int r = (blockIdx.x & 7) * 8 + warp;
     __nv_bfloat16* dst = out + ((int64_t)slot * SR_PAGE_ROWS + r) * d_model;
     __nv_bfloat16* cpy = copy_out ? copy_out + ((int64_t)slot * SR_PAGE_ROWS + r) * d_model : nullptr;
     if (r >= vr) {
@@ -229,13 +230,13 @@ sr_rmsnorm_rows_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, const __n
         ((uint4*)dst)[v] = make_uint4(0u, 0u, 0u, 0u);
         if (cpy) ((uint4*)cpy)[v] = make_uint4(0u, 0u, 0u, 0u);
       }
-      continue;
+      return;
     }
     const uint4* src;
     if (rows_in) {
       src = (const uint4*)(rows_in + ((int64_t)slot * SR_PAGE_ROWS + r) * d_model);
     } else {
-      if (!sr_check_page(s, s.slot_page[slot])) continue;
+      if (!sr_check_page(s, s.slot_page[slot])) return;
       src = (const uint4*)(pool.base + (int64_t)s.slot_page[slot] * pool.page_stride + (int64_t)pool_layer * pool.layer_stride +
                            (int64_t)r * pool.row_stride);
     }
@@ -327,6 +328,6 @@ cudaError_t sr_launch_rows_gemm(const SrSched& s, int kind, const __nv_bfloat16*
 cudaError_t sr_launch_rmsnorm_rows(const SrSched& s, const SrPoolView& pool, int32_t pool_layer, const __nv_bfloat16* rows_in,
                                    const __nv_bfloat16* w, float eps, int32_t d_model, __nv_bfloat16* out,
                                    __nv_bfloat16* copy_out, cudaStream_t stream) {
-  sr_rmsnorm_rows_kernel<<<(unsigned)s.max_slots, 256, 0, stream>>>(s, pool, pool_layer, rows_in, w, eps, d_model, out, copy_out);
+  sr_rmsnorm_rows_kernel<<<(unsigned)s.max_slots * 8, 256, 0, stream>>>(s, pool, pool_layer, rows_in, w, eps, d_model, out, copy_out);
   return cudaGetLastError();
 }
