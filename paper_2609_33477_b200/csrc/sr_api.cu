@@ -74,30 +74,6 @@ int check_pool(const sr_ctx* ctx, const sr_anchor_pool* p) {
   return SR_OK;
 }
 
-// Counts the kernel launches of one step and, when profiling is on, brackets them with two events on `stream`.
-struct LaunchScope {
-  sr_ctx* ctx;
-  cudaStream_t stream;
-  bool armed;
-  LaunchScope(sr_ctx* c, cudaStream_t s, int kind, int kernels = 1) : ctx(c), stream(s), armed(false) {
-    ctx->last_launches += kernels;
-    if (!ctx->profiling) return;
-    while (ctx->ev_pool.size() < ctx->ev_used + 2) {
-      cudaEvent_t e;
-      if (cudaEventCreate(&e) != cudaSuccess) return;
-      ctx->ev_pool.push_back(e);
-    }
-    if (cudaEventRecord(ctx->ev_pool[ctx->ev_used], stream) != cudaSuccess) return;
-    ctx->ev_kind.push_back(kind);
-    armed = true;
-  }
-  ~LaunchScope() {
-    if (!armed) return;
-    cudaEventRecord(ctx->ev_pool[ctx->ev_used + 1], stream);
-    ctx->ev_used += 2;
-  }
-};
-
 SrPoolView pool_view(const sr_anchor_pool* p) {
   SrPoolView v;
   v.base = (const char*)p->base;
@@ -309,7 +285,7 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
   if (sr_current_device_sms(&sm_count) != cudaSuccess) return SR_ERR_CUDA;
 
   {
-    LaunchScope scope(ctx, stream, SR_KERNEL_SCHEDULE);
+    SrLaunchScope scope(ctx, stream, SR_KERNEL_SCHEDULE);
     if (sr_launch_schedule(sched, table->pages, table->state_slots, replay_lens, table->max_pages,
                            table->max_replay_len, table->max_total_rows, pool->n_phys_pages, table->n_state_slots,
                            stream) != cudaSuccess)
@@ -359,7 +335,7 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
       if (hooks && !hooks->before(hooks->user, l, pl, ls)) break;
       if (in_conv) {
         __nv_bfloat16* hist = (__nv_bfloat16*)(base + lay.off_hist);
-        LaunchScope scope(ctx, ls, SR_KERNEL_CONV_TAIL);
+        SrLaunchScope scope(ctx, ls, SR_KERNEL_CONV_TAIL);
         if (sr_launch_hist_gather(ctx, sched, (const char*)in_conv->base + (int64_t)l * in_conv->layer_stride_bytes,
                                   in_conv->slot_stride_bytes, hist, ls) != cudaSuccess)
           break;
@@ -371,38 +347,38 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
       }
       if (ctx->fp16_stage) {
         {
-          LaunchScope scope(ctx, ls, SR_KERNEL_WEIGHT_DECODE);
+          SrLaunchScope scope(ctx, ls, SR_KERNEL_WEIGHT_DECODE);
           if (sr_launch_stage_weights_fp16(ctx, weights[l], (__half*)wdec, ls) != cudaSuccess) break;
         }
-        LaunchScope scope(ctx, ls, SR_KERNEL_ANCHOR_STAGE);
+        SrLaunchScope scope(ctx, ls, SR_KERNEL_ANCHOR_STAGE);
         if (sr_launch_stage_anchors_fp16(ctx, sched, pv, pl, (__half*)(base + lay.off_x16), ls) != cudaSuccess) break;
       } else if (ctx->w8a8) {
-        LaunchScope scope(ctx, ls, SR_KERNEL_ANCHOR_STAGE);
+        SrLaunchScope scope(ctx, ls, SR_KERNEL_ANCHOR_STAGE);
         if (sr_launch_quant_anchors_e4m3(ctx, sched, pv, pl, (uint8_t*)(base + lay.off_x16), (float*)(base + lay.off_sx), ls) !=
             cudaSuccess)
           break;
       } else if (ctx->wdec_bytes) {
-        LaunchScope scope(ctx, ls, SR_KERNEL_WEIGHT_DECODE);
+        SrLaunchScope scope(ctx, ls, SR_KERNEL_WEIGHT_DECODE);
         if (sr_launch_weight_decode(ctx, weights[l], wdec, ls) != cudaSuccess) break;
       }
       {
-        LaunchScope scope(ctx, ls, SR_KERNEL_PROJECTION, ctx->w8a8 ? 2 : 1);
+        SrLaunchScope scope(ctx, ls, SR_KERNEL_PROJECTION, ctx->w8a8 ? 2 : 1);
         if (sr_launch_proj_fused(ctx, sched, *pool, pl, weights[l], ctx->wdec_bytes ? wdec : nullptr, fused, sm_count,
                                  ls) != cudaSuccess)
           break;
       }
       {
-        LaunchScope scope(ctx, ls, SR_KERNEL_CONV_TAIL, sr_conv_tail_launches(ctx, sched.n_requests));
+        SrLaunchScope scope(ctx, ls, SR_KERNEL_CONV_TAIL, sr_conv_tail_launches(ctx, sched.n_requests));
         if (sr_launch_conv_tail(ctx, sched, pv, pl, weights[l], fused, conv_l, out_conv->slot_stride_bytes, ls) !=
             cudaSuccess)
           break;
       }
       {
-        LaunchScope scope(ctx, ls, SR_KERNEL_CHUNK_LOCAL);
+        SrLaunchScope scope(ctx, ls, SR_KERNEL_CHUNK_LOCAL);
         if (sr_launch_chunk_local(ctx, sched, weights[l], fused, split, ls) != cudaSuccess) break;
       }
       {
-        LaunchScope scope(ctx, ls, SR_KERNEL_SCAN);
+        SrLaunchScope scope(ctx, ls, SR_KERNEL_SCAN);
         if (sr_launch_scan_chain_umma(ctx, sched, fused, split, ssm_l, out_ssm->slot_stride_bytes, sm_count, ls) != cudaSuccess)
           break;
       }

@@ -47,6 +47,30 @@ struct sr_ctx {
   size_t ev_used;
 };
 
+// Counts the kernel launches of one step and, when profiling is on, brackets them with two events on `stream`.
+struct SrLaunchScope {
+  sr_ctx* ctx;
+  cudaStream_t stream;
+  bool armed;
+  SrLaunchScope(sr_ctx* c, cudaStream_t s, int kind, int kernels = 1) : ctx(c), stream(s), armed(false) {
+    ctx->last_launches += kernels;
+    if (!ctx->profiling) return;
+    while (ctx->ev_pool.size() < ctx->ev_used + 2) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      ctx->ev_pool.push_back(e);
+    }
+    if (cudaEventRecord(ctx->ev_pool[ctx->ev_used], stream) != cudaSuccess) return;
+    ctx->ev_kind.push_back(kind);
+    armed = true;
+  }
+  ~SrLaunchScope() {
+    if (!armed) return;
+    cudaEventRecord(ctx->ev_pool[ctx->ev_used + 1], stream);
+    ctx->ev_used += 2;
+  }
+};
+
 // Per-device one-time set-up (kernel attributes are per device, and several host threads may make their first
 // call at once): runs `setup` with the current device the first time `key` is seen on it, under a lock; later
 // calls return cudaSuccess at once.  A failed set-up is retried by the next call.

@@ -54,27 +54,6 @@ int check_group_ctx(const sr_ctx* ctx, const sr_page_table* t) {
   return SR_OK;
 }
 
-struct Scope {                      // counts launches; brackets them with events when profiling is on
-  sr_ctx* ctx; cudaStream_t stream; bool armed;
-  Scope(sr_ctx* c, cudaStream_t s, int kind) : ctx(c), stream(s), armed(false) {
-    ctx->last_launches += 1;
-    if (!ctx->profiling) return;
-    while (ctx->ev_pool.size() < ctx->ev_used + 2) {
-      cudaEvent_t e;
-      if (cudaEventCreate(&e) != cudaSuccess) return;
-      ctx->ev_pool.push_back(e);
-    }
-    if (cudaEventRecord(ctx->ev_pool[ctx->ev_used], stream) != cudaSuccess) return;
-    ctx->ev_kind.push_back(kind);
-    armed = true;
-  }
-  ~Scope() {
-    if (!armed) return;
-    cudaEventRecord(ctx->ev_pool[ctx->ev_used + 1], stream);
-    ctx->ev_used += 2;
-  }
-};
-
 }  // namespace
 
 extern "C" int sr_group_workspace_bytes(const sr_ctx* ctx, const sr_page_table* table, int32_t max_d_ff, size_t* out_bytes) {
@@ -181,7 +160,7 @@ extern "C" int sr_replay_group_states(sr_ctx* ctx, const sr_anchor_pool* pool, c
   xpool.layer_to_pool = pool->layer_to_pool;
 
   {
-    Scope scope(ctx, stream, SR_KERNEL_SCHEDULE);
+    SrLaunchScope scope(ctx, stream, SR_KERNEL_SCHEDULE);
     if (sr_launch_schedule(sched, table->pages, table->state_slots, replay_lens, table->max_pages, table->max_replay_len,
                            table->max_total_rows, pool->n_phys_pages, table->n_state_slots, stream) != cudaSuccess)
       return SR_ERR_CUDA;
@@ -196,26 +175,26 @@ extern "C" int sr_replay_group_states(sr_ctx* ctx, const sr_anchor_pool* pool, c
     {
       // layer input x = RMSNorm(r); the first layer reads the anchors through the page table and also leaves the
       // residual rows in packed order for the residual add
-      Scope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
+      SrLaunchScope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
       if (sr_launch_rmsnorm_rows(sched, pv, pl, j == 0 ? nullptr : r_cur, (const __nv_bfloat16*)b.norm_w, norm_eps, d.d_model, x,
                                  (j == 0 && !last) ? r_cur : nullptr, stream) != cudaSuccess)
         return SR_ERR_CUDA;
     }
     {
-      Scope scope(ctx, stream, SR_KERNEL_PROJECTION);
+      SrLaunchScope scope(ctx, stream, SR_KERNEL_PROJECTION);
       if (sr_launch_proj_fused(ctx, sched, xpool, 0, w, nullptr, fused, sm_count, stream) != cudaSuccess) return SR_ERR_CUDA;
     }
     {
-      Scope scope(ctx, stream, SR_KERNEL_CONV_TAIL);
+      SrLaunchScope scope(ctx, stream, SR_KERNEL_CONV_TAIL);
       if (sr_launch_conv_tail_from_raw(ctx, sched, fused, conv_l, out_conv->slot_stride_bytes, stream) != cudaSuccess)
         return SR_ERR_CUDA;
     }
     {
-      Scope scope(ctx, stream, SR_KERNEL_CHUNK_LOCAL);
+      SrLaunchScope scope(ctx, stream, SR_KERNEL_CHUNK_LOCAL);
       if (sr_launch_chunk_local(ctx, sched, w, fused, split, stream) != cudaSuccess) return SR_ERR_CUDA;
     }
     {
-      Scope scope(ctx, stream, SR_KERNEL_SCAN);
+      SrLaunchScope scope(ctx, stream, SR_KERNEL_SCAN);
       SrFused f2 = fused;
       if (last) { f2.dump_s = nullptr; f2.dump_u = nullptr; }
       if (sr_launch_scan_chain_umma(ctx, sched, f2, split, ssm_l, out_ssm->slot_stride_bytes, sm_count, stream) != cudaSuccess)
@@ -224,35 +203,35 @@ extern "C" int sr_replay_group_states(sr_ctx* ctx, const sr_anchor_pool* pool, c
     if (last) break;
     // output gate SiLU(x W_z^T), per-token outputs with head norm and gate, output projection + residual
     {
-      Scope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
+      SrLaunchScope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
       if (sr_launch_rows_gemm(sched, 1, x, dm, b.w_z, nullptr, (int32_t)hv, zg, hv, nullptr, 0, sm_count, stream) != cudaSuccess)
         return SR_ERR_CUDA;
     }
     {
-      Scope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
+      SrLaunchScope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
       if (sr_launch_group_output(ctx, sched, fused, split, zg, (const __nv_bfloat16*)b.o_norm_w, norm_eps, y, stream) != cudaSuccess)
         return SR_ERR_CUDA;
     }
     {
-      Scope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
+      SrLaunchScope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
       if (sr_launch_rows_gemm(sched, 2, y, hv, b.w_o, nullptr, d.d_model, r_nxt, dm, r_cur, dm, sm_count, stream) != cudaSuccess)
         return SR_ERR_CUDA;
     }
     __nv_bfloat16* t = r_cur; r_cur = r_nxt; r_nxt = t;
     if (b.mlp_norm_w) {
       {
-        Scope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
+        SrLaunchScope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
         if (sr_launch_rmsnorm_rows(sched, pv, 0, r_cur, (const __nv_bfloat16*)b.mlp_norm_w, norm_eps, d.d_model, x, nullptr, stream) !=
             cudaSuccess)
           return SR_ERR_CUDA;
       }
       {
-        Scope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
+        SrLaunchScope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
         if (sr_launch_rows_gemm(sched, 3, x, dm, b.w_gate, b.w_up, b.d_ff, hid, b.d_ff, nullptr, 0, sm_count, stream) != cudaSuccess)
           return SR_ERR_CUDA;
       }
       {
-        Scope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
+        SrLaunchScope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
         if (sr_launch_rows_gemm(sched, 2, hid, b.d_ff, b.w_down, nullptr, d.d_model, r_nxt, dm, r_cur, dm, sm_count, stream) != cudaSuccess)
           return SR_ERR_CUDA;
       }
