@@ -114,6 +114,16 @@ def test_a_group_of_one_layer_and_the_prefix_of_a_longer_group_agree():
     assert torch.equal(rep.out_ssm[:, :2], full_ssm[:, :2]) and torch.equal(rep.out_conv[:, :2], full_conv[:, :2])
     assert not rep.out_ssm[:, 2].any()                      # the third layer was not touched
     assert rep.last_launch_count() > 0
+    rep.out_ssm.zero_()
+    rep.out_conv.zero_()
+    rep.replay_group_states(first_layer=0, n_group_layers=1)    # a group of one: no block kernels at all
+    torch.cuda.synchronize()
+    assert rep.last_launch_count() == 6                     # packing + row norm, projection, conv state, chunk-local, chain
+    assert torch.equal(rep.out_ssm[:, 0], full_ssm[:, 0]) and torch.equal(rep.out_conv[:, 0], full_conv[:, 0])
+    assert not rep.out_ssm[:, 1:].any()
+    # a group must start at a layer that has anchors: layer 1 of this workload has none
+    assert rep.replay_group_states(first_layer=1, n_group_layers=2, check=False) == binding.SR_ERR_INVALID_ARG
+    assert rep.replay_group_states(first_layer=0, n_group_layers=4, check=False) == binding.SR_ERR_INVALID_ARG
 
 
 def test_group_at_the_benchmarked_size_matches_the_oracle_on_sampled_requests():
