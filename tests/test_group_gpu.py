@@ -208,3 +208,23 @@ def test_the_group_call_can_be_captured_in_a_cuda_graph():
     torch.cuda.synchronize()
     assert rep.group_device_status() == 0
     assert torch.equal(rep.out_ssm, ref_ssm) and torch.equal(rep.out_conv, ref_conv)
+
+
+def test_sentinel_requests_of_a_group_call_are_skipped_and_leave_the_others_unchanged():
+    """Destination slot -1 (Section 5.2, padded batches): nothing is written for that request, and the other requests
+    get the same bits as without it (rows of different requests never mix)."""
+    wl = synth.build_workload("group_small", device="cuda")
+    rep = binding.Replayer(wl)
+    rep.replay_group_states()
+    torch.cuda.synchronize()
+    ref_ssm, ref_conv = rep.out_ssm.clone(), rep.out_conv.clone()
+    slots = torch.tensor([0, 1, -1, 3], dtype=torch.int32, device="cuda")
+    rep2 = binding.Replayer(wl, state_slots=slots, n_slots=4)
+    rep2.out_ssm.fill_(7.0)
+    rep2.out_conv.fill_(7.0)
+    rep2.replay_group_states()
+    torch.cuda.synchronize()
+    assert rep2.group_device_status() == 0
+    for i in (0, 1, 3):
+        assert torch.equal(rep2.out_ssm[i], ref_ssm[i]) and torch.equal(rep2.out_conv[i], ref_conv[i])
+    assert (rep2.out_ssm[2] == 7.0).all() and (rep2.out_conv[2] == 7.0).all()
