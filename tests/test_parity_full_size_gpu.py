@@ -109,3 +109,16 @@ def test_cfg4_shorter_replay_lengths_of_the_sweep():
         print(f"{name}: worst rel Frobenius error per head {worst:.3e}")
         del wl, rep
         _free()
+
+
+def test_cfg4_w8a8_at_full_width_sampled_units():
+    """The 8-bit projection (quantised activations) at the benchmark's width and tile schedule: config 4 with 2048-row
+    windows (32 requests, 24 layers, d = 5120), two (request, layer) units against the W8A8 oracle."""
+    import dataclasses
+    spec = dataclasses.replace(synth.SPECS["cfg4_R2048"], name="cfg4_w8a8_R2048", act_quant="e4m3_1x128")
+    wl, rep = _run_full(spec)
+    _all_rebuilt_outputs_are_finite(wl, rep)
+    worst = _check_units(wl, rep, [(9, 3), (30, 22)])
+    print(f"cfg4_w8a8_R2048: worst rel Frobenius error per head over the sample {worst:.3e}")
+    del wl, rep
+    _free()
