@@ -67,3 +67,30 @@ def test_benchmark_specs_match_their_stated_shapes():
     assert (s["cfg2"].n_layers, s["cfg2"].d_model, s["cfg2"].conv_channels) == (48, 5120, 12288)
     assert s["cfg3"].layer_mask == "even" and s["cfg3"].n_requests == 64
     assert s["cfg4"].weight_format == "e4m3_block128" and abs(s["cfg4"].decay_scale - 0.03) < 1e-12
+
+
+def test_group_workloads_carry_block_weights_and_feed_the_oracle():
+    """Group workloads (Section 4.1): one pool layer holding the group-entry rows, every layer with mixer and block
+    weights; the fp64 images handed to the oracle are exact and the oracle runs on them."""
+    import numpy as np
+    from oracle import gdn_replay_oracle as orc
+    wl = synth.build_workload("group_small", device="cpu")
+    s = wl.spec
+    assert wl.anchor_pool.shape[1] == 1 and wl.layer_to_pool == [0, -1, -1] and wl.layer_mask == [1, 1, 1]
+    assert len(wl.blocks) == s.n_layers and all(p is not None for p in wl.layers)
+    assert [b.w_gate is not None for b in wl.blocks] == [False, True, False]          # d_ff = (0, 192, 0)
+    assert wl.blocks[1].w_gate.shape == (192, s.d_model) and wl.blocks[1].w_down.shape == (s.d_model, 192)
+    layers = [synth.block_arrays(wl.layers[l], wl.blocks[l]) for l in range(s.n_layers)]
+    assert np.array_equal(layers[0]["w_z"].astype(np.float32), wl.blocks[0].w_z.float().numpy())   # bf16 -> fp64 is exact
+    assert "w_gate" in layers[1] and "w_gate" not in layers[0]
+    i = 1
+    R = int(wl.replay_lens[i])
+    pages = wl.page_table[i, : -(-R // 64)].tolist()
+    got = synth.fetch_pages(wl, pages, 0)
+    rows = np.concatenate([orc.bf16_bits_to_f64(got[(p, 0)]) for p in pages])[:R]
+    res, handed = orc.group_replay(rows, layers, return_rows=True, n_k_heads=s.n_k_heads, n_v_heads=s.n_v_heads, d_k=s.d_k, d_v=s.d_v)
+    assert len(res) == 3 and len(handed) == 2 and handed[0].shape == (R, s.d_model)
+    assert all(np.all(np.isfinite(S)) and S.shape == (s.n_v_heads, s.d_k, s.d_v) for S, _ in res)
+    # same seed, same bytes
+    wl2 = synth.build_workload("group_small", device="cpu")
+    assert all(torch.equal(a.w_o, b.w_o) and torch.equal(a.norm_w, b.norm_w) for a, b in zip(wl.blocks, wl2.blocks))
