@@ -177,11 +177,11 @@ const char* sr_status_string(int status);
 
 /* Checks the geometry and builds a context (host memory only; no CUDA call).
  * Any consistent geometry (n_v_heads a multiple of n_k_heads) gets a context, so the size
- * queries below work for every model of Appendix A.  The kernels cover (d_k, d_v) in {(64, 64),
- * (128, 128), (96, 192)} -- the tensor-core scan and sr_replay_states_from only (128, 128), the
- * others run a token-by-token fp32 scan -- d_model % 128 == 0, conv_width == 4, page_rows == 64,
- * any n_v_heads = g * n_k_heads; for anything else sr_workspace_bytes,
- * sr_replay_states and sr_debug_gather return SR_ERR_UNSUPPORTED_SHAPE (there is no fallback). */
+ * queries below work for every model of Appendix A.  The kernels (one tensor-core path for every case) cover
+ * d_k in {64, 96, 128}, d_v a multiple of 8 with 2 d_k + d_v <= 512, any n_v_heads = g * n_k_heads with at most 128
+ * value heads, d_model a multiple of 64 (of 128 with block-scaled weights; with quantised activations H_k d_k and
+ * H_k d_k + H_v d_v must be multiples of 128 too), conv_width == 4, page_rows == 64; for anything else
+ * sr_workspace_bytes, sr_replay_states and sr_debug_gather return SR_ERR_UNSUPPORTED_SHAPE (there is no fallback). */
 int sr_create(const sr_model_desc* desc, sr_ctx** out_ctx);
 
 /* Frees a context.  NULL is allowed. */
@@ -278,9 +278,8 @@ int sr_replay_states_noalloc(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_p
  * `in_ssm`, `in_conv`: HOST structs describing DEVICE arrays with the layout and slot
  * addressing of the outputs (slot = state_slots[i] or i); either may be NULL (= zero).
  * Each may be the corresponding output array itself (states updated in place).  Requests
- * with replay length 0 hand their states through.  Only the default kernels serve this call
- * (d_k = d_v = 128 geometry): otherwise SR_ERR_UNSUPPORTED_SHAPE.  Everything else as
- * sr_replay_states.
+ * with replay length 0 hand their states through.  Served for every geometry sr_replay_states serves.
+ * Everything else as sr_replay_states.
  */
 int sr_replay_states_from(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* table,
                           const int32_t* replay_lens, const uint8_t* layer_mask,
