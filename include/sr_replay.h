@@ -25,7 +25,8 @@
  *   k = y_k / sqrt(sum y_k^2 + l2_eps) per (token, key head);  v = y_v;
  *   alpha = exp(-decay_scale[h] * softplus(a + dt_bias[h]));  beta = sigmoid(b);
  *   value head h uses key head h / (H_v / H_k).
- * Per-token outputs of the layer are never computed.
+ * Per-token outputs of the layer are never computed by sr_replay_states; sr_replay_group_states forms them to feed
+ * the next layer of a group.
  *
  * Conventions for every call
  *   - plain C types only; "DEVICE" marks pointers to GPU global memory, "HOST" host memory;
@@ -75,8 +76,9 @@ enum { SR_CONV_SILU = 0, SR_CONV_IDENTITY = 1 };  /* sr_model_desc.conv_activati
  * product up to fp32 summation and one 16-bit rounding of each weight.  E4M3_1X128 (W8A8, weight_format
  * SR_W_E4M3_BLOCK128 only): each anchor row is quantised on the fly, 128 channels at a time, s = max(amax, 1e-10)/448,
  * code = e4m3(x / s) (fp32, IEEE division, round to nearest even, saturating), and the products run on the 8-bit
- * tensor-core path at twice the 16-bit rate; a 128-deep partial sum enters the result as
- * weight scale x activation scale x partial sum in fp32.  The gate projection (bf16 weights) keeps the bf16 rows.
+ * tensor-core path; a 128-deep partial sum enters the result as weight scale x activation scale x partial sum in
+ * fp32, outside the tensor core -- which is what bounds this mode: with these plain fp32 scales it is the slower of
+ * the two on the benchmark configuration.  The gate projection (bf16 weights) keeps the bf16 rows.
  * W8A8 changes the VALUE computed (e4m3 keeps 4 significant bits of each activation): it is its own variant with
  * its own reference result, not an approximation of NONE held to the same tolerance. */
 enum { SR_AQ_NONE = 0, SR_AQ_E4M3_1X128 = 1 };
@@ -153,8 +155,8 @@ typedef struct sr_page_table {
   int32_t n_requests;          /* at most 65535 (one grid row per request), else SR_ERR_UNSUPPORTED_SHAPE */
   int32_t max_pages;           /* second extent of `pages` */
   int32_t max_replay_len;      /* upper bound on every replay_lens[i] (<= max_pages*page_rows) */
-  int64_t max_total_rows;      /* upper bound on the sum of replay_lens (sizes grid and workspace); with
-                                  d_k = d_v = 128 at most 65535 page slots per call, i.e.
+  int64_t max_total_rows;      /* upper bound on the sum of replay_lens (sizes grid and workspace); at most
+                                  65535 page slots per call (one grid row per slot), i.e.
                                   max_total_rows / 64 + n_requests <= 65535 (about 4.19 M rows), else
                                   SR_ERR_UNSUPPORTED_SHAPE */
   int32_t n_state_slots;       /* slots the output arrays hold, or 0 = not stated.  When stated, a destination
