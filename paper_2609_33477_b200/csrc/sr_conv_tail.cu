@@ -111,8 +111,8 @@ sr_conv_tail_kernel(SrSched s, SrPoolView pool, int32_t pool_layer, int32_t d_mo
 }
 
 // Channels as one GEMM over the batch: out[r][c] = sum_k X[r][k] W[c][k] for the gathered tail rows r = 3 i + j
-// (request i, window entry j).  One CTA = 64 rows x 64 channels, four warps of 16 rows each, k in chunks of 64 through
-// a four-stage ring (cp.async for the anchor rows and for bf16 weights).  Rows without a source (before a request's
+// (request i, window entry j).  One CTA = 64 rows x 64 channels, four warps (each owns 16 channels for every 16-row block), k in chunks of 64
+// through a four-stage ring (cp.async for the anchor rows and for bf16 weights).  Rows without a source (before a request's
 // first token, past the batch, skipped requests) read some valid row and are masked on output.
 //   FP8 = false: bf16 weights, the q channels only (k, v rows come from the projection).
 //   FP8 = true : e4m3 codes with 128 x 128 block scales, every channel q | k | v.  The bare codes are decoded to
