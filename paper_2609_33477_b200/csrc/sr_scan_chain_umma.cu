@@ -30,6 +30,9 @@
 // W^T and U~^T do not depend on the state: they are issued one chunk ahead (behind the previous chunk's state
 // update, as soon as tensor memory for them is drained), and the key tiles are double-buffered so that loads
 // run two chunks ahead.  On the serial chain remain: drain S and W^T, S^T W^T, drain U^T, the state update.
+// For group-propagated replay (Section 4.1) the passes that drain S and U^T also leave the fp16 state ENTERING
+// every chunk and the chunk's U^T (before the row factors) in memory: the output kernel forms the layer's per-token
+// outputs from them.
 // Every mbarrier wait is bounded; on expiry the kernel raises SR_DEV_WAIT_EXPIRED, stops issuing work,
 // frees its tensor memory and returns.
 #include "sr_umma.cuh"
