@@ -308,6 +308,23 @@ def run_group(args, wl, dev, rank, world, warmup):
         t, n = binding.sr_profile_read(rep.ctx, kind)
         kernel_ms[k] = {"ms": t, "launches": n} if n else None
     binding.sr_profile_enable(rep.ctx, False)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # the oracle on the host cores: the whole group for the first request (a fixed, bounded job)
+        import numpy as np
+        from oracle import gdn_replay_oracle as orc
+        from paper_2609_33477_b200 import synth
+        R0 = int(wl.replay_lens[0].item())
+        pages = wl.page_table[0, : -(-R0 // 64)].cpu().tolist()
+        got = synth.fetch_pages(wl, pages, 0)
+        rows0 = np.concatenate([orc.bf16_bits_to_f64(got[(p, 0)]) for p in pages])[:R0]
+        layers = [synth.block_arrays(wl.layers[l], wl.blocks[l]) for l in range(spec.n_layers)]
+        t0 = time.perf_counter()
+        orc.group_replay(rows0, layers, n_k_heads=spec.n_k_heads, n_v_heads=spec.n_v_heads, d_k=spec.d_k, d_v=spec.d_v)
+        dt = time.perf_counter() - t0
+        cpu_baseline = {"value": R0 * spec.n_layers / dt, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
+                        "sample": f"{spec.name}: request 0 ({R0} rows), all {spec.n_layers} layers of the group, once",
+                        "seconds": dt}
     hv = spec.n_v_heads * spec.d_v
     L = spec.n_layers
     proj = L * 2.0 * spec.d_model * (spec.conv_channels + 2 * spec.n_v_heads)
@@ -330,7 +347,7 @@ def run_group(args, wl, dev, rank, world, warmup):
                          "frac": (proj + block) * rows / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                          "peak_source": f"{peaks['source']} bf16 burst", "traffic": None, "kernel_ms": kernel_ms,
                          "block_tflops": (block * rows / (gb["ms"] * 1e-3) / 1e12) if gb else None},
-            "cpu_baseline": None}), flush=True)
+            "cpu_baseline": cpu_baseline}), flush=True)
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
