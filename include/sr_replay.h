@@ -198,7 +198,7 @@ int sr_conv_bytes_per_layer(const sr_ctx* ctx, size_t* out_bytes);
 /* Scratch bytes sr_replay_states should be given for any batch within the bounds in `table`
  * (n_requests, max_pages, max_total_rows; the pointers in `table` are not read).  The layers of one call are
  * independent of one another (every layer has its own anchors, Eq. 2), so for a batch too small to fill the GPU
- * with one layer the call runs up to four layers side by side, each with its own block of scratch: this size
+ * with one layer the call runs up to eight layers side by side, each with its own block of scratch: this size
  * includes those blocks (as many as stay within 1 GiB together; one block for large batches, where keeping a
  * second layer in flight under the first one's projection measured within +-2 % of running them in turn). */
 int sr_workspace_bytes(const sr_ctx* ctx, const sr_page_table* table, size_t* out_bytes);

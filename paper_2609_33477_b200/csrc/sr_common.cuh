@@ -15,7 +15,7 @@
 
 #define SR_PAGE_ROWS 64
 #define SR_CONV_W 4
-#define SR_MAX_LANES 4                       // layers in flight at once on small batches
+#define SR_MAX_LANES 8                       // layers in flight at once on small batches
 #define SR_LANES_BUDGET_BYTES (1024ull << 20) // ... as long as their hand-over buffers together stay below this
 
 struct sr_ctx {
@@ -37,8 +37,8 @@ struct sr_ctx {
   std::vector<cudaEvent_t> ev_pool;   // created on demand, reused, destroyed with the context
   // small batches: layers are independent, so up to SR_MAX_LANES of them run side by side on streams of the
   // context (lane 0 is the caller's stream); created at the first call that uses them
-  cudaStream_t lane_stream[3];
-  cudaEvent_t lane_fork, lane_join[3];
+  cudaStream_t lane_stream[SR_MAX_LANES - 1];
+  cudaEvent_t lane_fork, lane_join[SR_MAX_LANES - 1];
   bool lanes_ready;
   // sr_replay_states_host only: two copy streams and their events, created at its first call
   cudaStream_t copy_in, copy_out;

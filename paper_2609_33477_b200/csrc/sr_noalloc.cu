@@ -49,7 +49,7 @@ extern "C" int sr_replay_states_noalloc(sr_ctx* ctx, const sr_anchor_pool* pool,
   int st = sr_workspace_bytes(ctx, table, &need);       // checks `ctx` and the bounds in `table`
   if (st != SR_OK) return st;
   // what the call cannot do without: the tables and ONE block of per-layer hand-over buffers (sr_workspace_bytes
-  // asks for up to four blocks on small batches, to run layers side by side; this entry uses as many as fit).
+  // asks for up to eight blocks on small batches, to run layers side by side; this entry uses as many as fit).
   // If even that is more than the fixed array holds: refuse, launch nothing.
   need = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, 1).total;
   if (need > (size_t)SR_NOALLOC_SCRATCH_BYTES) return SR_ERR_WORKSPACE;

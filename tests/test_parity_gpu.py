@@ -332,7 +332,7 @@ def test_second_forms_match_oracle(flag, name):
 
 def test_layers_run_side_by_side_with_the_same_bits_as_one_after_the_other():
     """A small batch with nine rebuilt layers: with the recommended workspace the call spreads the layers over
-    four streams of the context, with the minimum workspace it runs them in order.  Same bits either way, and
+    several streams of the context, with the minimum workspace it runs them in order.  Same bits either way, and
     both match the oracle."""
     wl = synth.build_workload("layers_small", device=DEV)
     wide = B.Replayer(wl)
