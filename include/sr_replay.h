@@ -359,7 +359,9 @@ int sr_group_workspace_bytes(const sr_ctx* ctx, const sr_page_table* table, int3
  * bf16 weights (SR_W_BF16) and (d_k, d_v) in {(64, 64), (128, 128)}, d_model and H_v*d_v multiples of 64;
  * else SR_ERR_UNSUPPORTED_SHAPE.  `debug_rows`: NULL, or DEVICE bf16 [n_group_layers - 1][max_slots * 64][d_model]
  * receiving the rows handed from each layer to the next in packed page-slot order (request i's rows start at page
- * slot sum_{i' < i} ceil(R_i' / 64)); a test aid.  Asynchronous on `stream`, no allocation, no host sync.
+ * slot sum_{i' < i} ceil(R_i' / 64)); a test aid.  Asynchronous on `stream`, no allocation, no host sync.  One
+ * kernel per layer (the output gate) runs on a stream of the context that forks from `stream` and joins it again, so
+ * the call stays one unit of work on `stream`; the first call creates that stream: make it outside any stream capture.
  */
 int sr_replay_group_states(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* table,
                            const int32_t* replay_lens, int32_t first_layer, int32_t n_group_layers,

@@ -236,8 +236,10 @@ int validate_call(const sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_t
   return SR_OK;
 }
 
+}  // namespace
+
 // the context's lane streams and their fork / join events, made once
-bool ensure_lanes(sr_ctx* ctx) {
+bool sr_ensure_lanes(sr_ctx* ctx) {
   if (ctx->lanes_ready) return true;
   for (int i = 0; i < SR_MAX_LANES - 1; ++i) {
     if (cudaStreamCreateWithFlags(&ctx->lane_stream[i], cudaStreamNonBlocking) != cudaSuccess) return false;
@@ -247,6 +249,8 @@ bool ensure_lanes(sr_ctx* ctx) {
   ctx->lanes_ready = true;
   return true;
 }
+
+namespace {
 
 int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* table, const int32_t* replay_lens,
                 const uint8_t* layer_mask, const sr_layer_weights* weights, const sr_out* out_ssm,
@@ -274,7 +278,7 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
                        sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, lanes).total > workspace_bytes))
     lanes >>= 1;
   const SrWorkspace lay = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, lanes);
-  if (lanes > 1 && !ensure_lanes(ctx)) return SR_ERR_CUDA;
+  if (lanes > 1 && !sr_ensure_lanes(ctx)) return SR_ERR_CUDA;
 
   SrSched sched = sr_sched_view(workspace, lay, table->n_requests);
   sched.check_bounds = (ctx->debug_flags & SR_DEBUG_CHECK_BOUNDS) ? 1 : 0;

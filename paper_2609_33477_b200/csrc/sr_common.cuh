@@ -82,6 +82,8 @@ enum SrOnceKey {
 cudaError_t sr_once_per_device(int key, cudaError_t (*setup)());
 // SM count of the current device (looked up once per device)
 cudaError_t sr_current_device_sms(int* sms);
+// Creates the context's side streams and fork / join events at first use (outside any stream capture).
+bool sr_ensure_lanes(sr_ctx* ctx);
 
 // Scratch layout inside the caller's workspace (all offsets in bytes, 256-aligned).
 struct sr_ctx;

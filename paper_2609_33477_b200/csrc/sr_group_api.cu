@@ -107,6 +107,7 @@ extern "C" int sr_replay_group_states(sr_ctx* ctx, const sr_anchor_pool* pool, c
   if (table->n_requests == 0) return SR_OK;
   int sm_count = 0;
   if (sr_current_device_sms(&sm_count) != cudaSuccess) return SR_ERR_CUDA;
+  const bool side = n_group_layers > 1 && sr_ensure_lanes(ctx);
 
   char* ws = (char*)workspace;
   SrSched sched = sr_sched_view(workspace, lay.base, table->n_requests);
@@ -184,6 +185,24 @@ extern "C" int sr_replay_group_states(sr_ctx* ctx, const sr_anchor_pool* pool, c
       SrLaunchScope scope(ctx, stream, SR_KERNEL_PROJECTION);
       if (sr_launch_proj_fused(ctx, sched, xpool, 0, w, nullptr, fused, sm_count, stream) != cudaSuccess) return SR_ERR_CUDA;
     }
+    if (side && !last) {
+      // The output gate SiLU(x W_z^T) needs only x: it runs on a side stream of the context next to the conv-state,
+      // chunk-local and chain kernels, which leave most of the GPU idle on a serving-size batch; the caller's stream
+      // waits for it before the per-token outputs.
+      cudaStream_t ss = ctx->lane_stream[0];
+      if (cudaEventRecord(ctx->lane_fork, stream) != cudaSuccess || cudaStreamWaitEvent(ss, ctx->lane_fork, 0) != cudaSuccess)
+        return SR_ERR_CUDA;
+      cudaError_t e;
+      {
+        SrLaunchScope scope(ctx, ss, SR_KERNEL_GROUP_BLOCK);
+        e = sr_launch_rows_gemm(sched, 1, x, dm, b.w_z, nullptr, (int32_t)hv, zg, hv, nullptr, 0, sm_count, ss);
+      }
+      // joined whatever happened, so the call stays one unit of work on `stream`
+      if (cudaEventRecord(ctx->lane_join[0], ss) != cudaSuccess || e != cudaSuccess) {
+        cudaStreamWaitEvent(stream, ctx->lane_join[0], 0);
+        return SR_ERR_CUDA;
+      }
+    }
     {
       SrLaunchScope scope(ctx, stream, SR_KERNEL_CONV_TAIL);
       if (sr_launch_conv_tail_from_raw(ctx, sched, fused, conv_l, out_conv->slot_stride_bytes, stream) != cudaSuccess)
@@ -201,12 +220,15 @@ extern "C" int sr_replay_group_states(sr_ctx* ctx, const sr_anchor_pool* pool, c
         return SR_ERR_CUDA;
     }
     if (last) break;
-    // output gate SiLU(x W_z^T), per-token outputs with head norm and gate, output projection + residual
-    {
+    if (side) {
+      if (cudaStreamWaitEvent(stream, ctx->lane_join[0], 0) != cudaSuccess) return SR_ERR_CUDA;
+    } else {
+      // output gate SiLU(x W_z^T)
       SrLaunchScope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
       if (sr_launch_rows_gemm(sched, 1, x, dm, b.w_z, nullptr, (int32_t)hv, zg, hv, nullptr, 0, sm_count, stream) != cudaSuccess)
         return SR_ERR_CUDA;
     }
+    // per-token outputs with head norm and gate, output projection + residual
     {
       SrLaunchScope scope(ctx, stream, SR_KERNEL_GROUP_BLOCK);
       if (sr_launch_group_output(ctx, sched, fused, split, zg, (const __nv_bfloat16*)b.o_norm_w, norm_eps, y, stream) != cudaSuccess)
