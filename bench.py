@@ -29,11 +29,12 @@ UNIT = "layer-tokens/s"
 DEFAULT_CONFIG = "cfg3"
 
 # Where the DRAM traffic of the dominant kernel comes from: the committed summary of an ncu capture of that
-# kernel on a slice of the workload (same kernel, tile shapes and per-row traffic, small enough to capture).
+# kernel -- at full size where the two DRAM counters fit one ncu pass (cfg3), else on a slice of the workload (same
+# kernel, tile shapes and per-row traffic, small enough to capture).
 # Each summary carries one line `traffic_per_launch: read_bytes=... write_bytes=... rows=...`; the figure
 # reported here is that capture scaled by rows (an upper bound: the weight part of the reads does not grow).
 NCU_TRAFFIC_SUMMARY = {
-    "cfg3": "sr_proj_fused2_kernel_cfg3_slice.md", "cfg3_slice": "sr_proj_fused2_kernel_cfg3_slice.md",
+    "cfg3": "dram_traffic_cfg3_full.md", "cfg3_slice": "sr_proj_fused2_kernel_cfg3_slice.md",
     "cfg2": "sr_proj_fused2_kernel_cfg3_slice.md",
     "cfg4": "sr_proj_fused2_kernel_fp8_cfg4_slice.md", "cfg4_slice": "sr_proj_fused2_kernel_fp8_cfg4_slice.md",
 }
@@ -56,6 +57,8 @@ def ncu_traffic(config, rows):
         return None, None
     cap_rows = int(m.group(3))
     total = float(m.group(1)) + float(m.group(2))
+    if cap_rows == rows:
+        return total, f"profiles/{name} (captured at this size, {rows} rows)"
     return total * rows / cap_rows, f"profiles/{name} ({cap_rows} rows captured, scaled by rows to {rows})"
 
 
