@@ -35,8 +35,8 @@ DEFAULT_CONFIG = "cfg3"
 # reported here is that capture scaled by rows (an upper bound: the weight part of the reads does not grow).
 NCU_TRAFFIC_SUMMARY = {
     "cfg3": "dram_traffic_cfg3_full.md", "cfg3_slice": "sr_proj_fused2_kernel_cfg3_slice.md",
-    "cfg2": "sr_proj_fused2_kernel_cfg3_slice.md",
-    "cfg4": "sr_proj_fused2_kernel_fp8_cfg4_slice.md", "cfg4_slice": "sr_proj_fused2_kernel_fp8_cfg4_slice.md",
+    "cfg2": "dram_traffic_cfg3_full.md", "cfg4": "dram_traffic_cfg3_full.md",
+    "cfg4_slice": "sr_proj_fused2_kernel_fp8_cfg4_slice.md",
 }
 
 
@@ -52,7 +52,8 @@ def ncu_traffic(config, rows):
         text = open(path).read()
     except OSError:
         return None, None
-    m = re.search(r"traffic_per_launch:\s*read_bytes=([0-9.eE+]+)\s+write_bytes=([0-9.eE+]+)\s+rows=(\d+)", text)
+    pat = r"\s*read_bytes=([0-9.eE+]+)\s+write_bytes=([0-9.eE+]+)\s+rows=(\d+)"
+    m = re.search("traffic_per_launch_" + config + ":" + pat, text) or re.search("traffic_per_launch:" + pat, text)
     if not m:
         return None, None
     cap_rows = int(m.group(3))
