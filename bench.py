@@ -34,10 +34,10 @@ DEFAULT_CONFIG = "cfg3"
 # Each summary carries one line `traffic_per_launch: read_bytes=... write_bytes=... rows=...`; the figure
 # reported here is that capture scaled by rows (an upper bound: the weight part of the reads does not grow).
 NCU_TRAFFIC_SUMMARY = {
-    "cfg3": "dram_traffic_cfg3_full.md", "cfg3_slice": "sr_proj_fused2_kernel_cfg3_slice.md",
-    "cfg2": "dram_traffic_cfg3_full.md", "cfg4": "dram_traffic_cfg3_full.md",
-    "cfg4_slice": "sr_proj_fused2_kernel_fp8_cfg4_slice.md",
+    "cfg3_slice": "sr_proj_fused2_kernel_cfg3_slice.md", "cfg4_slice": "sr_proj_fused2_kernel_fp8_cfg4_slice.md",
 }
+NCU_TRAFFIC_SUMMARY.update({c: "dram_traffic_full_size.md" for c in
+                            ("cfg0", "cfg1", "cfg2", "cfg3", "cfg4", "cfg4_w8a8", "hit_512", "hits8_512")})
 
 
 def ncu_traffic(config, rows):
