@@ -228,3 +228,17 @@ def test_sentinel_requests_of_a_group_call_are_skipped_and_leave_the_others_unch
     for i in (0, 1, 3):
         assert torch.equal(rep2.out_ssm[i], ref_ssm[i]) and torch.equal(rep2.out_conv[i], ref_conv[i])
     assert (rep2.out_ssm[2] == 7.0).all() and (rep2.out_conv[2] == 7.0).all()
+
+
+def test_group_call_under_device_side_bounds_checks_raises_no_alarm():
+    """SR_DEBUG_CHECK_BOUNDS: every table-driven index is tested before the access; a healthy call sets no bit and
+    gives the same bits as without the checks."""
+    wl = synth.build_workload("group_small", device="cuda")
+    rep = binding.Replayer(wl)
+    rep.replay_group_states()
+    torch.cuda.synchronize()
+    chk = binding.Replayer(wl, debug_flags=binding.SR_DEBUG_CHECK_BOUNDS)
+    chk.replay_group_states()
+    torch.cuda.synchronize()
+    assert chk.group_device_status() == 0
+    assert torch.equal(chk.out_ssm, rep.out_ssm) and torch.equal(chk.out_conv, rep.out_conv)
