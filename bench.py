@@ -285,8 +285,13 @@ def run_group(args, wl, dev, rank, world, warmup):
     rep = binding.Replayer(wl)
     stream = torch.cuda.current_stream(dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    groups = wl.groups
+    if len(groups) > 1:          # all the model's groups in one call, side by side
+        call = lambda: rep.replay_groups_states(stream=stream)
+    else:
+        call = lambda: rep.replay_group_states(stream=stream)
     for _ in range(warmup):
-        rep.replay_group_states(stream=stream)
+        call()
     torch.cuda.synchronize(dev)
     assert rep.group_device_status() == 0
     launches = rep.last_launch_count()
@@ -297,15 +302,26 @@ def run_group(args, wl, dev, rank, world, warmup):
     for i in range(args.steps):
         flush.fill_(i & 0xFF)
         e0.record(stream)
-        rep.replay_group_states(stream=stream)
+        call()
         e1.record(stream)
         torch.cuda.synchronize(dev)
         times.append(e0.elapsed_time(e1))
     clocks = sampler.stop()
+    in_turn_ms = None
+    if len(groups) > 1:          # the same groups one after the other (the least workspace)
+        seq = []
+        for i in range(min(args.steps, 5)):
+            flush.fill_(i & 0xFF)
+            e0.record(stream)
+            rep.replay_groups_states(stream=stream, min_workspace=True)
+            e1.record(stream)
+            torch.cuda.synchronize(dev)
+            seq.append(e0.elapsed_time(e1))
+        in_turn_ms = sorted(seq)[len(seq) // 2]
     total_ms = max_over_ranks(sum(times), dev)
     ms = total_ms / args.steps
     binding.sr_profile_enable(rep.ctx, True)
-    rep.replay_group_states(stream=stream)
+    call()
     torch.cuda.synchronize(dev)
     kernel_ms = {}
     for k, kind in binding.KERNEL_KINDS.items():
@@ -332,7 +348,9 @@ def run_group(args, wl, dev, rank, world, warmup):
     hv = spec.n_v_heads * spec.d_v
     L = spec.n_layers
     proj = L * 2.0 * spec.d_model * (spec.conv_channels + 2 * spec.n_v_heads)
-    block = (L - 1) * 4.0 * spec.d_model * hv + sum(6.0 * spec.d_model * f for f in spec.d_ff[:L - 1])
+    block = 0.0                  # every layer but the last of each group runs its block
+    for first, n in groups:
+        block += (n - 1) * 4.0 * spec.d_model * hv + sum(6.0 * spec.d_model * f for f in spec.d_ff[first:first + n - 1])
     rows = wl.total_rows
     peaks = measured_peaks()
     gb = kernel_ms.get("group_block")
@@ -341,7 +359,8 @@ def run_group(args, wl, dev, rank, world, warmup):
             "metric": METRIC, "value": world * rows * L / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": spec.name, "group_layers": L, "d_model": spec.d_model, "heads": spec.n_v_heads,
+            "config": {"workload": spec.name, "group_layers": L, "groups": len(groups), "groups_in_turn_ms": in_turn_ms,
+                       "d_model": spec.d_model, "heads": spec.n_v_heads,
                        "d_head": spec.d_k, "d_ff": list(spec.d_ff), "requests": spec.n_requests, "replayed_rows": rows,
                        "l2": "256 MB flush buffer written between timed steps"},
             "clocks": clocks, "e2e": None, "gpu_launches": launches * args.steps,

@@ -370,6 +370,25 @@ int sr_replay_group_states(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_pag
                            size_t workspace_bytes, void* stream);
 
 /*
+ * Several groups in one call: group g covers layers first_layers[g] .. first_layers[g] + group_sizes[g] - 1 (HOST arrays
+ * of n_groups entries; the groups must not overlap), each replayed from its own group-entry anchors exactly as
+ * sr_replay_group_states does it -- same kernels, same bits.  The groups are independent (Section 4.1: each group
+ * restarts from its own anchor), so the call keeps several of them in flight, each on a stream of the context with
+ * its own block of scratch: as many as sr_groups_workspace_bytes made room for (up to eight, within 1 GiB together), or
+ * as fit the workspace given (at least sr_group_workspace_bytes: then one group after the other).  The streams fork
+ * from `stream` after the batch is packed and join it before the call's work ends (the first call creates them: make
+ * it outside any stream capture).  This is the form a cache hit on a hybrid model takes: all its linear-attention
+ * groups at once.
+ */
+int sr_groups_workspace_bytes(const sr_ctx* ctx, const sr_page_table* table, int32_t max_d_ff, int32_t n_groups,
+                              size_t* out_bytes);
+int sr_replay_groups_states(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* table,
+                            const int32_t* replay_lens, int32_t n_groups, const int32_t* first_layers,
+                            const int32_t* group_sizes, const sr_layer_weights* weights, const sr_block_weights* blocks,
+                            float norm_eps, const sr_out* out_ssm, const sr_out* out_conv, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
+/*
  * The write side of the sidecar (Section 5.1, "Writing anchors": the host precomputes a
  * destination table for the step; indexed copies inside the step's graph write the selected
  * hidden states directly to their sidecar locations; unsampled positions receive a scratch

@@ -32,7 +32,8 @@ EXPORTS = (
     "sr_conv_bytes_per_layer", "sr_workspace_bytes", "sr_replay_states", "sr_replay_states_host",
     "sr_debug_gather", "sr_device_status", "sr_last_launch_count", "sr_profile_enable", "sr_profile_read",
     "sr_replay_states_noalloc", "sr_replay_states_from", "sr_anchor_write", "sr_workspace_bytes_min",
-    "sr_debug_quantise", "sr_group_workspace_bytes", "sr_replay_group_states",
+    "sr_debug_quantise", "sr_group_workspace_bytes", "sr_replay_group_states", "sr_groups_workspace_bytes",
+    "sr_replay_groups_states",
 )
 SR_NOALLOC_SCRATCH_BYTES = 128 * 1024 * 1024
 SR_KERNEL_SCHEDULE, SR_KERNEL_PROJECTION, SR_KERNEL_CONV_TAIL, SR_KERNEL_SCAN = 0, 1, 2, 3
@@ -128,6 +129,11 @@ def load() -> C.CDLL:
         C.c_void_p, C.POINTER(sr_anchor_pool), C.POINTER(sr_page_table), C.c_void_p, C.c_int32, C.c_int32,
         C.POINTER(sr_layer_weights), C.POINTER(sr_block_weights), C.c_float, C.POINTER(sr_out), C.POINTER(sr_out),
         C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sr_groups_workspace_bytes.argtypes = [C.c_void_p, C.POINTER(sr_page_table), C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]
+    lib.sr_replay_groups_states.argtypes = [
+        C.c_void_p, C.POINTER(sr_anchor_pool), C.POINTER(sr_page_table), C.c_void_p, C.c_int32, C.POINTER(C.c_int32),
+        C.POINTER(C.c_int32), C.POINTER(sr_layer_weights), C.POINTER(sr_block_weights), C.c_float, C.POINTER(sr_out),
+        C.POINTER(sr_out), C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sr_device_status.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_uint32)]
     lib.sr_last_launch_count.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
     lib.sr_profile_enable.argtypes = [C.c_void_p, C.c_int]
@@ -194,6 +200,21 @@ def sr_group_workspace_bytes(ctx, table: sr_page_table, max_d_ff: int) -> int:
     out = C.c_size_t()
     _check(load().sr_group_workspace_bytes(ctx, C.byref(table), int(max_d_ff), C.byref(out)), "sr_group_workspace_bytes")
     return int(out.value)
+
+
+def sr_groups_workspace_bytes(ctx, table: sr_page_table, max_d_ff: int, n_groups: int) -> int:
+    out = C.c_size_t()
+    _check(load().sr_groups_workspace_bytes(ctx, C.byref(table), int(max_d_ff), int(n_groups), C.byref(out)),
+           "sr_groups_workspace_bytes")
+    return int(out.value)
+
+
+def sr_replay_groups_states(ctx, pool, table, replay_lens_ptr, first_layers: Sequence[int], group_sizes: Sequence[int], weights,
+                            blocks, norm_eps, out_ssm, out_conv, workspace_ptr, workspace_bytes, stream_ptr) -> int:
+    n = len(first_layers)
+    return load().sr_replay_groups_states(ctx, C.byref(pool), C.byref(table), replay_lens_ptr, n, (C.c_int32 * n)(*first_layers),
+                                          (C.c_int32 * n)(*group_sizes), weights, blocks, float(norm_eps), C.byref(out_ssm),
+                                          C.byref(out_conv), workspace_ptr, workspace_bytes, stream_ptr)
 
 
 def sr_replay_group_states(ctx, pool, table, replay_lens_ptr, first_layer, n_group_layers, weights, blocks, norm_eps,
@@ -380,17 +401,7 @@ class Replayer:
         if wl.blocks is None:
             raise ValueError("not a group workload")
         g = spec.n_layers - first_layer if n_group_layers is None else int(n_group_layers)
-        if not hasattr(self, "_blocks"):
-            self._blocks = (sr_block_weights * spec.n_layers)()
-            ptr = lambda t: t.data_ptr() if t is not None else None
-            for l, b in enumerate(wl.blocks):
-                self._blocks[l] = sr_block_weights(ptr(b.norm_w), ptr(b.w_z), ptr(b.o_norm_w), ptr(b.w_o), ptr(b.mlp_norm_w),
-                                                   ptr(b.w_gate), ptr(b.w_up), ptr(b.w_down),
-                                                   int(b.w_gate.shape[0]) if b.w_gate is not None else 0)
-            max_ff = max([int(b.w_gate.shape[0]) for b in wl.blocks if b.w_gate is not None] + [0])
-            self._group_ws_bytes = sr_group_workspace_bytes(self.ctx, self.table, max_ff)
-            self._group_ws = torch.empty(self._group_ws_bytes + 256, dtype=torch.uint8, device=self.device)
-            self._group_ws_ptr = (self._group_ws.data_ptr() + 255) // 256 * 256
+        self._group_setup()
         rows = None
         if debug_rows and g > 1:
             B = self.table.n_requests
@@ -403,6 +414,41 @@ class Replayer:
         if check:
             _check(st, "sr_replay_group_states")
         return (st, rows) if debug_rows else st
+
+    def _group_setup(self, n_groups: int = 1) -> None:
+        """Block-weight structs and a workspace with room for ``n_groups`` groups side by side (made once, grown on demand)."""
+        wl, spec = self.wl, self.spec
+        if not hasattr(self, "_blocks"):
+            self._blocks = (sr_block_weights * spec.n_layers)()
+            ptr = lambda t: t.data_ptr() if t is not None else None
+            for l, b in enumerate(wl.blocks):
+                self._blocks[l] = sr_block_weights(ptr(b.norm_w), ptr(b.w_z), ptr(b.o_norm_w), ptr(b.w_o), ptr(b.mlp_norm_w),
+                                                   ptr(b.w_gate), ptr(b.w_up), ptr(b.w_down),
+                                                   int(b.w_gate.shape[0]) if b.w_gate is not None else 0)
+            self._max_ff = max([int(b.w_gate.shape[0]) for b in wl.blocks if b.w_gate is not None] + [0])
+            self._group_ws_bytes = 0
+        need = sr_groups_workspace_bytes(self.ctx, self.table, self._max_ff, n_groups)
+        if need > self._group_ws_bytes:
+            self._group_ws_bytes = need
+            self._group_ws = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+            self._group_ws_ptr = (self._group_ws.data_ptr() + 255) // 256 * 256
+
+    def replay_groups_states(self, groups: Optional[Sequence] = None, norm_eps: float = 1e-6, stream=None, check: bool = True,
+                             min_workspace: bool = False) -> int:
+        """One ``sr_replay_groups_states`` call: ``groups`` = [(first_layer, n_layers), ...] (default: the workload's own
+        groups), replayed side by side where the workspace has room (``min_workspace``: one group's worth only)."""
+        wl = self.wl
+        if wl.blocks is None:
+            raise ValueError("not a group workload")
+        groups = list(wl.groups) if groups is None else list(groups)
+        self._group_setup(1 if min_workspace else len(groups))
+        ws_bytes = sr_group_workspace_bytes(self.ctx, self.table, self._max_ff) if min_workspace else self._group_ws_bytes
+        st = sr_replay_groups_states(self.ctx, self.pool, self.table, wl.replay_lens.data_ptr(), [g[0] for g in groups],
+                                     [g[1] for g in groups], self.weights, self._blocks, norm_eps, self._out_ssm, self._out_conv,
+                                     self._group_ws_ptr, ws_bytes, self._stream_ptr(stream))
+        if check:
+            _check(st, "sr_replay_groups_states")
+        return st
 
     def group_device_status(self, stream=None) -> int:
         return sr_device_status(self.ctx, self._group_ws_ptr, self._stream_ptr(stream))

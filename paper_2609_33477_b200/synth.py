@@ -56,6 +56,7 @@ class WorkloadSpec:
     # only anchors are the rows entering layer 0; every layer gets block weights, and an MLP d_ff[l] wide (0: none)
     group: bool = False
     d_ff: Tuple = ()
+    group_size: int = 0               # layers per group (0: all n_layers are one group); anchors enter each group's first layer
 
     @property
     def conv_channels(self) -> int:
@@ -147,6 +148,15 @@ SPECS["group_128"] = WorkloadSpec(name="group_128", n_layers=2, d_model=512, n_k
                                   n_requests=2, replay=("list", (300, 64)), group=True, d_ff=(512, 0))
 SPECS["group_wide"] = WorkloadSpec(name="group_wide", n_layers=2, d_model=640, n_k_heads=1, n_v_heads=3, d_k=128, d_v=128,
                                    n_requests=3, replay=("list", (129, 1, 257)), group=True, d_ff=(448, 0))
+# a cache hit on a hybrid model: all its linear-attention groups at once (Section 4.1; the 3 : 1 pattern gives groups of
+# three) -- 24 layers of the 4B geometry in eight groups, MLPs behind every layer, one 512-anchor hit / eight of them
+SPECS["groups8_hit_512"] = WorkloadSpec(name="groups8_hit_512", n_layers=24, d_model=2560, n_k_heads=16, n_v_heads=32, d_k=128,
+                                        d_v=128, n_requests=1, replay=("fixed", 512), group=True, group_size=3,
+                                        d_ff=(10240,) * 24)
+SPECS["groups8_hits8_512"] = dataclasses.replace(SPECS["groups8_hit_512"], name="groups8_hits8_512", n_requests=8)
+SPECS["groups_small"] = WorkloadSpec(name="groups_small", n_layers=7, d_model=256, n_k_heads=2, n_v_heads=4, d_k=64, d_v=64,
+                                     n_requests=3, replay=("list", (70, 0, 200)), group=True, group_size=3,
+                                     d_ff=(0, 192, 0, 128, 0, 0, 64))
 SPECS["group3_4b"] = WorkloadSpec(name="group3_4b", n_layers=3, d_model=2560, n_k_heads=16, n_v_heads=32, d_k=128, d_v=128,
                                   n_requests=8, replay=("fixed", 512), group=True, d_ff=(10240, 10240, 10240))
 for _r in (1024, 2048, 4096):
@@ -187,6 +197,12 @@ class Workload:
     replay_lens: torch.Tensor           # [B] int32, rows to replay per request
     layers: List[Optional[LayerParams]]  # None for masked-out layers
     blocks: Optional[List[BlockParams]] = None   # group workloads only
+
+    @property
+    def groups(self) -> List[Tuple[int, int]]:
+        """(first layer, layers) of every group of a group workload."""
+        gs = self.spec.group_size or self.spec.n_layers
+        return [(f, min(gs, self.spec.n_layers - f)) for f in range(0, self.spec.n_layers, gs)]
 
     @property
     def n_phys_pages(self) -> int:
@@ -302,8 +318,12 @@ def build_workload(spec_or_name, device="cpu", seed: int = 0,
     layer_to_pool, n_pool = [], 0
     for l in range(spec.n_layers):
         if spec.group:                 # one anchor per group: the rows entering its first layer
-            layer_to_pool.append(0 if l == 0 else -1)
-            n_pool = 1
+            gs = spec.group_size or spec.n_layers
+            if l % gs == 0:
+                layer_to_pool.append(n_pool)
+                n_pool += 1
+            else:
+                layer_to_pool.append(-1)
         elif mask[l]:
             layer_to_pool.append(n_pool)
             n_pool += 1

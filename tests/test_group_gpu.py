@@ -59,13 +59,15 @@ def _strict_conv(tail_gpu, tail_ref):
     assert ((dist <= 1) | (np.abs(a - b) <= 1e-5)).all() and (dist > 0).mean() <= 0.02
 
 
-def _oracle_group(wl, i):
+def _oracle_group(wl, i, first=0, n=None):
     s = wl.spec
+    n = s.n_layers - first if n is None else n
+    pl = wl.layer_to_pool[first]
     R = int(wl.replay_lens[i].item())
     pages = wl.page_table[i, : -(-R // 64)].cpu().tolist()
-    got = synth.fetch_pages(wl, pages, 0)
-    rows = np.concatenate([orc.bf16_bits_to_f64(got[(p, 0)]) for p in pages])[:R] if R else np.zeros((0, s.d_model))
-    layers = [synth.block_arrays(wl.layers[l], wl.blocks[l]) for l in range(s.n_layers)]
+    got = synth.fetch_pages(wl, pages, pl)
+    rows = np.concatenate([orc.bf16_bits_to_f64(got[(p, pl)]) for p in pages])[:R] if R else np.zeros((0, s.d_model))
+    layers = [synth.block_arrays(wl.layers[l], wl.blocks[l]) for l in range(first, first + n)]
     return orc.group_replay(rows, layers, return_rows=True, n_k_heads=s.n_k_heads, n_v_heads=s.n_v_heads, d_k=s.d_k, d_v=s.d_v)
 
 
@@ -242,3 +244,38 @@ def test_group_call_under_device_side_bounds_checks_raises_no_alarm():
     torch.cuda.synchronize()
     assert chk.group_device_status() == 0
     assert torch.equal(chk.out_ssm, rep.out_ssm) and torch.equal(chk.out_conv, rep.out_conv)
+
+
+
+def test_several_groups_in_one_call_match_the_oracle_and_the_single_group_calls():
+    """sr_replay_groups_states: the groups of a hybrid model side by side, each from its own anchors (Section 4.1)."""
+    wl = synth.build_workload("groups_small", device="cuda")
+    s = wl.spec
+    assert wl.groups == [(0, 3), (3, 3), (6, 1)] and wl.anchor_pool.shape[1] == 3
+    rep = binding.Replayer(wl)
+    rep.replay_groups_states()
+    torch.cuda.synchronize()
+    assert rep.group_device_status() == 0
+    all_ssm, all_conv = rep.out_ssm.clone(), rep.out_conv.clone()
+    for i in range(s.n_requests):
+        for first, n in wl.groups:
+            res, _ = _oracle_group(wl, i, first, n)
+            for j, (S_ref, tail_ref) in enumerate(res):
+                err = U.rel_frob_per_head(all_ssm[i, first + j].cpu().numpy(), S_ref)
+                assert err <= U.REL_FROB_TOL + 1e-2 * j, f"request {i} group at {first} layer {j}: {err:.3e}"
+                if j == 0:
+                    _strict_conv(_bits(all_conv[i, first]), tail_ref)
+    # the same bits one group at a time, and with the least workspace (groups one after the other)
+    rep.out_ssm.zero_()
+    rep.out_conv.zero_()
+    for first, n in wl.groups:
+        rep.replay_group_states(first_layer=first, n_group_layers=n)
+    torch.cuda.synchronize()
+    assert torch.equal(rep.out_ssm, all_ssm) and torch.equal(rep.out_conv, all_conv)
+    rep.out_ssm.zero_()
+    rep.out_conv.zero_()
+    rep.replay_groups_states(min_workspace=True)
+    torch.cuda.synchronize()
+    assert torch.equal(rep.out_ssm, all_ssm) and torch.equal(rep.out_conv, all_conv)
+    # overlapping groups are refused on the host
+    assert rep.replay_groups_states(groups=[(0, 3), (2, 2)], check=False) == binding.SR_ERR_INVALID_ARG
