@@ -279,3 +279,22 @@ def test_several_groups_in_one_call_match_the_oracle_and_the_single_group_calls(
     assert torch.equal(rep.out_ssm, all_ssm) and torch.equal(rep.out_conv, all_conv)
     # overlapping groups are refused on the host
     assert rep.replay_groups_states(groups=[(0, 3), (2, 2)], check=False) == binding.SR_ERR_INVALID_ARG
+
+
+def test_the_multi_group_call_can_be_captured_in_a_cuda_graph():
+    """The side streams fork from and join the capturing stream, so the whole call becomes one graph."""
+    wl = synth.build_workload("groups_small", device="cuda")
+    rep = binding.Replayer(wl)
+    rep.replay_groups_states()                       # creates the side streams and the workspace, outside the capture
+    torch.cuda.synchronize()
+    ref_ssm, ref_conv = rep.out_ssm.clone(), rep.out_conv.clone()
+    rep.out_ssm.zero_()
+    rep.out_conv.zero_()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        rep.replay_groups_states(stream=torch.cuda.current_stream())
+    graph.replay()
+    torch.cuda.synchronize()
+    assert rep.group_device_status() == 0
+    assert torch.equal(rep.out_ssm, ref_ssm) and torch.equal(rep.out_conv, ref_conv)
