@@ -7,18 +7,19 @@
 // serves the output gate (x W_z^T, SiLU applied), the output projection (y W_o^T + residual), and the two MLP
 // products (SiLU(n W_gate^T) * (n W_up^T), then ... W_down^T + residual).  tcgen05 tensor cores, tokens on the
 // MMA's M axis (a tensor-memory lane is a row, so a thread writes consecutive output columns of its row):
-// persistent, one CTA per SM, warp 0 TMA producer (128 rows of A and 256 rows of B per 64-wide k block, 4-stage
-// ring), warp 1 MMA issuer with a double-buffered accumulator (2 x 256 columns of tensor memory), warps 2-5
-// epilogue.  All waits are bounded.
+// persistent, CTAs paired into clusters of two that share one 256 x 256 MMA tile (cta_group::2); per CTA warp 0 is
+// the TMA producer (its 128 rows of A and its 128 of the tile's 256 weight rows per 64-wide k block, 6-stage ring),
+// warp 1 of the leader issues the MMAs into a double-buffered accumulator (2 x 256 columns of tensor memory per
+// CTA), warps 2-5 are the epilogue.  All waits are bounded.
 #include "sr_umma.cuh"
 
 namespace {
 
-constexpr int GM = 128;                  // rows per tile (MMA M): two page slots
-constexpr int GN = 256;                  // output columns per tile (MMA N)
-constexpr int GK = 64, GSTAGES = 4;
-constexpr int GA_BYTES = GM * GK * 2;    // 16 KB
-constexpr int GB_BYTES = GN * GK * 2;    // 32 KB
+constexpr int GM = 128;                  // rows per CTA (a pair of CTAs works on 256 rows: four page slots)
+constexpr int GN = 256;                  // output columns per tile (MMA N); each CTA of the pair stages 128 weight rows
+constexpr int GK = 64, GSTAGES = 6;
+constexpr int GA_BYTES = GM * GK * 2;          // 16 KB: this CTA's 128 rows
+constexpr int GB_BYTES = (GN / 2) * GK * 2;    // 16 KB: this CTA's 128 of the tile's 256 weight rows
 constexpr int GSTAGE_BYTES = GA_BYTES + GB_BYTES;
 constexpr int GSMEM_BYTES = GSTAGES * GSTAGE_BYTES + 1024 + 256;
 constexpr int GTHREADS = 192;
@@ -39,37 +40,46 @@ enum { EPI_STORE = 0, EPI_SILU = 1, EPI_ADD = 2, EPI_SWIGLU = 3 };
 
 __device__ __forceinline__ float silu(float x) { return __fdividef(x, 1.f + __expf(-x)); }
 
+// Two-CTA form (tcgen05 cta_group::2), as in the in-projection: a pair of CTAs on neighbouring SMs shares one MMA
+// tile of 256 rows x 256 columns.  Each CTA stages its own 128 rows and 128 of the tile's 256 weight rows per k
+// block (32 KB) and the tensor core reads the weight operand from both shared memories: a weight tile crosses from
+// L2 once per 256 rows instead of once per 128, which is what bounds these products on a serving-size batch (a few
+// hundred rows against hundreds of megabytes of weights).  The leader CTA issues the MMAs; both CTAs run their own
+// TMA producer and their own epilogue (their 128 rows of the accumulator).
 template <int EPI>
-__global__ void __launch_bounds__(GTHREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GTHREADS, 1)
 sr_rows_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_b2, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint64_t* full_bar = (uint64_t*)(smem + GSTAGES * GSTAGE_BYTES);
-  uint64_t* empty_bar = full_bar + GSTAGES;
-  uint64_t* tfull_bar = empty_bar + GSTAGES;
-  uint64_t* tempty_bar = tfull_bar + 2;
+  uint64_t* full_bar = (uint64_t*)(smem + GSTAGES * GSTAGE_BYTES);   // used in the leader CTA only
+  uint64_t* empty_bar = full_bar + GSTAGES;                          // one set per CTA
+  uint64_t* tfull_bar = empty_bar + GSTAGES;                         // [2] one set per CTA
+  uint64_t* tempty_bar = tfull_bar + 2;                              // [2] used in the leader CTA only
   uint32_t* tmem_slot = (uint32_t*)(tempty_bar + 2);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int n_slots = (int)p.s.status[1];
-  const int m_tiles = (n_slots + 1) / 2;
+  const int m_tiles = (n_slots + 3) / 4;
   const long long total_tiles = (long long)m_tiles * p.n_tiles;
   constexpr int NCOL = EPI == EPI_SWIGLU ? GN / 2 : GN;      // output columns a tile produces
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < GSTAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&tfull_bar[i], 1); mbar_init(&tempty_bar[i], 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&tfull_bar[i], 1); mbar_init(&tempty_bar[i], 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  cluster_sync_all();               // the partner's barriers exist before anything signals them
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
@@ -85,42 +95,42 @@ sr_rows_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     mt = r / nbt;
     nt = blk * p.n_block + r % nbt;
   };
+  // does the second CTA's half of the weight tile exist?  (Both CTAs and the leader's byte count must agree.)
+  auto second_half = [&](int nt) { return EPI == EPI_SWIGLU || nt * GN + GN / 2 < p.n; };
 
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      for (long long tile = pair; ok && tile < total_tiles; tile += n_pairs) {
         int mt, nt;
         tile_coords(tile, mt, nt);
+        const bool second = second_half(nt);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
           uint8_t* a_dst = smem + stage * GSTAGE_BYTES;
           uint8_t* b_dst = a_dst + GA_BYTES;
-          // the second half of the weight tile is fetched only where the matrix has rows for it: what the MMA then
-          // reads there is stale shared memory, and the accumulator columns it feeds are never stored
-          const bool second = EPI == EPI_SWIGLU || nt * GN + GN / 2 < p.n;
-          mbar_expect_tx(&full_bar[stage], second ? GSTAGE_BYTES : GSTAGE_BYTES - GB_BYTES / 2);
-          tma_load_2d(a_dst, &map_a, &full_bar[stage], kb * GK, mt * GM);
-          if (EPI == EPI_SWIGLU) {       // 128 gate rows, then the 128 up rows of the same hidden units
-            tma_load_2d(b_dst, &map_b, &full_bar[stage], kb * GK, nt * NCOL);
-            tma_load_2d(b_dst + GB_BYTES / 2, &map_b2, &full_bar[stage], kb * GK, nt * NCOL);
-          } else {
-            tma_load_2d(b_dst, &map_b, &full_bar[stage], kb * GK, nt * GN);
-            if (second) tma_load_2d(b_dst + GB_BYTES / 2, &map_b, &full_bar[stage], kb * GK, nt * GN + GN / 2);
+          // both CTAs' loads land on the leader's barrier; a missing second half is stale shared memory whose
+          // accumulator columns are never stored
+          if (rank == 0) mbar_expect_tx(&full_bar[stage], second ? 2 * GSTAGE_BYTES : 2 * GSTAGE_BYTES - GB_BYTES);
+          tma_load_2d_pair(a_dst, &map_a, &full_bar[stage], kb * GK, (2 * mt + rank) * GM);
+          if (EPI == EPI_SWIGLU) {       // columns 0..127: gate rows (CTA 0), 128..255: the up rows of the same hidden units
+            tma_load_2d_pair(b_dst, rank == 0 ? &map_b : &map_b2, &full_bar[stage], kb * GK, nt * NCOL);
+          } else if (rank == 0 || second) {
+            tma_load_2d_pair(b_dst, &map_b, &full_bar[stage], kb * GK, nt * GN + rank * (GN / 2));
           }
           if (++stage == GSTAGES) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      const uint32_t idesc = umma_idesc(GM, GN);
-      for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      const uint32_t idesc = umma_idesc(2 * GM, GN);
+      for (long long tile = pair; ok && tile < total_tiles; tile += n_pairs) {
         if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag, p.s.status)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * GN;
@@ -131,24 +141,24 @@ sr_rows_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const uint64_t a_desc = umma_smem_desc(a_addr), b_desc = umma_smem_desc(a_addr + GA_BYTES);
 #pragma unroll
           for (int k = 0; k < GK / 16; ++k)
-            umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
-          umma_commit(&empty_bar[stage]);
+            umma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_commit_pair(&empty_bar[stage]);          // frees the stage in both CTAs
           if (++stage == GSTAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(&tfull_bar[acc]);
+        umma_commit_pair(&tfull_bar[acc]);              // accumulator complete, in both CTAs
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
   } else {
-    // epilogue: thread = row (tensor-memory lane 32 * (warp % 4) + lane)
+    // epilogue: thread = row (tensor-memory lane 32 * (warp % 4) + lane) of this CTA's 128 rows
     const int quarter = warp & 3;
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (long long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    for (long long tile = pair; tile < total_tiles; tile += n_pairs) {
       int mt, nt;
       tile_coords(tile, mt, nt);
-      const long long row = (long long)mt * GM + quarter * 32 + lane;
+      const long long row = (long long)(2 * mt + rank) * GM + quarter * 32 + lane;
       const bool row_ok = row < (long long)n_slots * SR_PAGE_ROWS && sr_check_slot(p.s, (int)(row / SR_PAGE_ROWS));
       if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag, p.s.status)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -196,16 +206,17 @@ sr_rows_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+      if (lane == 0) mbar_arrive_leader(&tempty_bar[acc]);
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }
 
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  cluster_sync_all();               // neither CTA leaves (or frees tensor memory) while the other may still signal it
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
   }
 }
 
@@ -271,9 +282,10 @@ bool encode_rows(CUtensorMap* map, const void* base, uint64_t k, uint64_t rows, 
 template <int EPI>
 cudaError_t launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mb2, const GemmParams& p,
                         long long max_tiles, int sm_count, cudaStream_t stream) {
-  int grid = (int)(max_tiles < sm_count ? max_tiles : sm_count);
-  if (grid < 1) grid = 1;
-  sr_rows_gemm_kernel<EPI><<<grid, GTHREADS, GSMEM_BYTES, stream>>>(ma, mb, mb2, p);
+  long long pairs = sm_count / 2;
+  if (max_tiles < pairs) pairs = max_tiles;
+  if (pairs < 1) pairs = 1;
+  sr_rows_gemm_kernel<EPI><<<(unsigned)(2 * pairs), GTHREADS, GSMEM_BYTES, stream>>>(ma, mb, mb2, p);
   return cudaGetLastError();
 }
 
@@ -315,7 +327,8 @@ cudaError_t sr_launch_rows_gemm(const SrSched& s, int kind, const __nv_bfloat16*
   p.ldc = ldc;
   p.residual = residual;
   p.ldr = ldr;
-  const long long max_tiles = (long long)((s.max_slots + 1) / 2) * p.n_tiles;
+  if (sm_count < 2) return cudaErrorNotSupported;
+  const long long max_tiles = (long long)((s.max_slots + 3) / 4) * p.n_tiles;
   switch (kind) {
     case EPI_STORE: return launch_gemm<EPI_STORE>(ma, mb, mb2, p, max_tiles, sm_count, stream);
     case EPI_SILU: return launch_gemm<EPI_SILU>(ma, mb, mb2, p, max_tiles, sm_count, stream);
