@@ -334,43 +334,57 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 // W8A8: e4m3 weight codes (as the caller stores them) x e4m3 activation codes (written by the quantiser, page-slot
 // order), tcgen05 kind::f8f6f4, one 128-byte row of K per stage.  Both operands carry block scales that are plain
 // fp32 numbers, not the hardware's power-of-two block format, so every 128-deep K group has to enter the result as
-//     total[channel][token] += w_scale[channel block][group] * x_scale[token][group] * partial[channel][token]
-// outside the tensor core: one multiply-add per output element per group, which is what bounds this kernel.
+//     total[token][channel] += w_scale[channel block][group] * x_scale[token][group] * partial[token][channel]
+// outside the tensor core: one multiply-add per output element per group.  To make that fold cost nothing but the
+// multiply-add, this kernel puts the TOKENS on the MMA's M axis (128 tokens = two page slots; N = 256 channels =
+// two 128-channel scale blocks): a tensor-memory lane -- a thread -- is then a token, a warpgroup owns one scale
+// block, and the scale product of a group is ONE number per thread, fetched two groups ahead.
 // Layout: three warpgroups.  Warpgroup 0 holds the TMA producer and the MMA issuer and gives most of its registers
-// away (setmaxnreg); warpgroups 1 and 2 take them and keep the TOTALS IN REGISTERS -- a thread owns one channel
-// (tensor-memory lane) and 128 tokens, warpgroup 1 the tile's first two page slots, warpgroup 2 the other two.  The
-// partial sums of a group (128 channels x 256 tokens, one MMA of N = 256 per 32 codes of K) are double-buffered in
-// tensor memory (2 x 256 columns), so the tensor core works on group g + 1 while the warpgroups fold group g.  After
-// the last group the conv + SiLU epilogue runs straight from the registers (every slot's first three rows are
-// finished later by the chunk-local kernel, like the first rows of a tile in the 16-bit kernels).
+// away (setmaxnreg); warpgroups 1 and 2 take them and keep the TOTALS IN REGISTERS (one token x 128 channels per
+// thread), while the partial sums of a group are double-buffered in tensor memory (2 x 256 columns), so the tensor
+// core works on group g + 1 while group g is folded.  The waits on that short chain (group done -> fold -> buffer
+// free -> next group) poll instead of suspending.
+// The conv + SiLU epilogue wants the other orientation (a thread walks the tokens of one channel): after the last
+// group each warpgroup turns its totals around through shared memory, 64 channels at a time -- every thread writes
+// its token's totals as a column, then reads one channel's 64 tokens of one page slot as a row -- and the epilogue
+// of the 16-bit kernels runs unchanged (every slot's first three rows are finished later by the chunk-local kernel,
+// like the first rows of a tile in the 16-bit kernels).
 constexpr int W8_BK = 128;                       // bytes (= codes) of K per stage
 constexpr int W8_THREADS = 384;
-constexpr int W8_SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + 2 * 2 * BN * 4;
+constexpr int W8_TOK = 128;                      // tokens per tile (MMA M)
+constexpr int W8_SLOTS = W8_TOK / SR_PAGE_ROWS;
+constexpr int W8_CH = 256;                       // channels per tile (MMA N)
+constexpr int W8_STAGES = 3;
+constexpr int W8_X_BYTES = W8_TOK * W8_BK;       // 16 KB of activation codes
+constexpr int W8_W_BYTES = W8_CH * W8_BK;        // 32 KB of weight codes
+constexpr int W8_STAGE_BYTES = W8_X_BYTES + W8_W_BYTES;
+constexpr int W8_TR_LD = W8_TOK + 4;             // floats per channel row of a turn-around buffer (bank spread)
+constexpr int W8_TR_BYTES = 64 * W8_TR_LD * 4;   // 64 channels x 128 tokens per warpgroup and round
+constexpr int W8_SMEM_BYTES = W8_STAGES * W8_STAGE_BYTES + 2 * W8_TR_BYTES + 1024 + 256;
 
 __global__ void __launch_bounds__(W8_THREADS, 1)
 sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const FusedParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint64_t* full_bar = (uint64_t*)(smem + STAGES * STAGE_BYTES);
-  uint64_t* empty_bar = full_bar + STAGES;
-  uint64_t* pfull_bar = empty_bar + STAGES;      // [2] partial sums of a group complete in buffer b
-  uint64_t* pempty_bar = pfull_bar + 2;          // [2] ... folded into the totals by the eight epilogue warps
-  uint64_t* sx_full = pempty_bar + 2;            // [2] activation scales of a K group landed
-  uint32_t* tmem_slot = (uint32_t*)(sx_full + 2);
+  float* turn = (float*)(smem + W8_STAGES * W8_STAGE_BYTES);     // [2 warpgroups][64][W8_TR_LD]
+  uint64_t* full_bar = (uint64_t*)(smem + W8_STAGES * W8_STAGE_BYTES + 2 * W8_TR_BYTES);
+  uint64_t* empty_bar = full_bar + W8_STAGES;
+  uint64_t* pfull_bar = empty_bar + W8_STAGES;   // [2] partial sums of a group complete in buffer b
+  uint64_t* pempty_bar = pfull_bar + 2;          // [2] ... folded into the totals by the eight folding warps
+  uint32_t* tmem_slot = (uint32_t*)(pempty_bar + 2);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
-  float* sxs = (float*)(smem + STAGES * STAGE_BYTES + 256);      // [2][BN] activation scales of a K group
-  float* comb = sxs + 2 * BN;                                    // [2][BN] weight scale x activation scale
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_slots = (int)p.s.status[1];
-  const int t_tiles = (n_slots + SLOTS - 1) / SLOTS;
-  const int c_tiles = p.n_ct;                    // the bf16 gate rows go through their own launch
+  const int t_tiles = (n_slots + W8_SLOTS - 1) / W8_SLOTS;
+  const int c_tiles = (p.n_ct + 1) / 2;          // 256-channel tiles of k | v (the last may be half empty); the bf16
+                                                 // gate rows go through their own launch
   const long long total_tiles = (long long)t_tiles * c_tiles;
   const int k_groups = p.k_blocks;               // one stage = one 128-deep group
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&pfull_bar[i], 1); mbar_init(&pempty_bar[i], 8); mbar_init(&sx_full[i], 1); }
+    for (int i = 0; i < W8_STAGES; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&pfull_bar[i], 1); mbar_init(&pempty_bar[i], 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -383,19 +397,8 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  auto tile_coords = [&](long long tile, int& ct, int& tt) {     // same walk as the 16-bit kernels
-    const long long per_group = (long long)p.group_t * c_tiles;
-    const int g = (int)(tile / per_group);
-    int r = (int)(tile % per_group);
-    const int gt = min(p.group_t, t_tiles - g * p.group_t);
-    const int per_block = gt * p.group_c;
-    const int cb = r / per_block;
-    r -= cb * per_block;
-    const int gc = min(p.group_c, c_tiles - cb * p.group_c);
-    ct = cb * p.group_c + r % gc;
-    tt = g * p.group_t + r / gc;
-  };
-
+  // Tile order: channel-fastest.  The 8-bit k | v weights of a layer (tens of MB) stay in L2 as a whole; the CTAs
+  // work on a handful of neighbouring token tiles at a time, whose codes are read from HBM once.
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
     if (warp == 0 && lane == 0) {                // TMA producer
@@ -403,126 +406,132 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
       uint32_t phase = 0;
       bool ok = true;
       for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        int ct, tt;
-        tile_coords(tile, ct, tt);
+        const int tt = (int)(tile / c_tiles), ct = (int)(tile % c_tiles);
         for (int kb = 0; kb < k_groups; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
-          uint8_t* a_dst = smem + stage * STAGE_BYTES;
-          uint8_t* b_dst = a_dst + A_BYTES;
-          mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
-          tma_load_2d(a_dst, &map_w, &full_bar[stage], kb * W8_BK, p.w_row0 + ct * BM);
+          uint8_t* x_dst = smem + stage * W8_STAGE_BYTES;
+          uint8_t* w_dst = x_dst + W8_X_BYTES;
+          mbar_expect_tx(&full_bar[stage], W8_STAGE_BYTES);
 #pragma unroll
-          for (int q = 0; q < SLOTS; ++q)
-            tma_load_4d(b_dst + q * (B_BYTES / SLOTS), &map_x, &full_bar[stage], kb * W8_BK, 0, 0, SLOTS * tt + q);
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          for (int q = 0; q < W8_SLOTS; ++q)
+            tma_load_4d(x_dst + q * (W8_X_BYTES / W8_SLOTS), &map_x, &full_bar[stage], kb * W8_BK, 0, 0, W8_SLOTS * tt + q);
+#pragma unroll
+          for (int h = 0; h < 2; ++h)            // rows past the weight matrix arrive as zeros
+            tma_load_2d(w_dst + h * (W8_W_BYTES / 2), &map_w, &full_bar[stage], kb * W8_BK, p.w_row0 + ct * W8_CH + h * BM);
+          if (++stage == W8_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
     } else if (warp == 1 && lane == 0) {         // MMA issue
       int stage = 0;
       uint32_t phase = 0, gcount = 0;
       bool ok = true;
-      const uint32_t idesc = umma_idesc_e4m3(BM, BN);
+      const uint32_t idesc = umma_idesc_e4m3(W8_TOK, W8_CH);
       for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        int ct, tt;
-        tile_coords(tile, ct, tt);
         for (int kg = 0; kg < k_groups; ++kg, ++gcount) {
           const uint32_t b = gcount & 1u;
-          // buffer b was folded two groups ago: its partial sums and its scale buffer are free
-          if (!mbar_wait(&pempty_bar[b], ((gcount >> 1) & 1u) ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
+          // buffer b was folded two groups ago
+          if (!mbar_wait_spin(&pempty_bar[b], ((gcount >> 1) & 1u) ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
+          if (!mbar_wait_spin(&full_bar[stage], phase, abort_flag, p.s.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          mbar_expect_tx(&sx_full[b], BN * 4);   // this group's activation scales: one 64-float run per page slot
-#pragma unroll
-          for (int q = 0; q < SLOTS; ++q)
-            bulk_load(sxs + b * BN + q * SR_PAGE_ROWS, p.sx + ((long long)(SLOTS * tt + q) * k_groups + kg) * SR_PAGE_ROWS,
-                      SR_PAGE_ROWS * 4, &sx_full[b]);
-          if (!mbar_wait(&full_bar[stage], phase, abort_flag, p.s.status)) { ok = false; break; }
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t a_addr = smem_u32(smem + stage * STAGE_BYTES);
-          const uint64_t a_desc = umma_smem_desc(a_addr), b_desc = umma_smem_desc(a_addr + A_BYTES);
+          const uint32_t x_addr = smem_u32(smem + stage * W8_STAGE_BYTES);
+          const uint64_t a_desc = umma_smem_desc(x_addr), b_desc = umma_smem_desc(x_addr + W8_X_BYTES);
 #pragma unroll
           for (int k = 0; k < W8_BK / 32; ++k)
-            umma_e4m3(tmem_base + b * (uint32_t)BN, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, k != 0 ? 1u : 0u);
+            umma_e4m3(tmem_base + b * (uint32_t)W8_CH, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, k != 0 ? 1u : 0u);
           umma_commit(&pfull_bar[b]);
           umma_commit(&empty_bar[stage]);
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          if (++stage == W8_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
-    // epilogue: tensor-memory lanes 32 * (warp % 4) .., tokens wg * 128 .. + 127 of the tile
+    // fold: tensor-memory lanes 32 * (warp % 4) .. = tokens of the tile, columns wg * 128 .. + 127 = channels
     const int quarter = warp & 3, wg = (warp >> 2) - 1;
-    const int ch_local = quarter * 32 + lane;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    const int e = wg * 128 + (warp & 3) * 32 + lane;       // this thread's entry of the scale products
+    float* buf = turn + wg * (W8_TR_BYTES / 4);
+    const int tid = quarter * 32 + lane;                   // the token while folding; (slot, channel) = (tid / 64, tid % 64) after
+    const int last_block = (p.n_q + p.n_kv - 1) / 128;     // last row of the weight-scale matrix
     uint32_t gcount = 0;
     bool ok = true;
-    for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-      int ct, tt;
-      tile_coords(tile, ct, tt);
-      const int ch = ct * BM + ch_local;
-      const float* scale_row = p.w_scale + (long long)((p.n_q + ct * BM) / 128) * p.scale_ld;
+    for (long long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const int tt = (int)(tile / c_tiles), ct = (int)(tile % c_tiles);
+      const int cb = 2 * ct + wg;                          // this warpgroup's 128-channel block of k | v
+      const float* ws = p.w_scale + (long long)min((p.n_q + cb * BM) / 128, last_block) * p.scale_ld;
+      const float* xs = p.sx + (long long)(W8_SLOTS * tt + (tid >> 6)) * k_groups * SR_PAGE_ROWS + (tid & 63);
+      // what the epilogue will need, fetched before the K loop
+      const int sl = tid >> 6, slot = W8_SLOTS * tt + sl;
+      const int vr = p.s.slot_rows[slot], first = p.s.slot_first[slot];
+      uint2 cwv[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int ch = cb * BM + r * 64 + (tid & 63);
+        cwv[r] = ch < p.n_kv ? __ldg((const uint2*)(p.conv_w + (long long)(p.n_q + ch) * SR_CONV_W)) : make_uint2(0u, 0u);
+      }
       float tot[128];
 #pragma unroll
       for (int i = 0; i < 128; ++i) tot[i] = 0.f;
+      // the scales of group kg + 2 are fetched while group kg is folded
+      float w_cur = __ldg(ws), x_cur = __ldg(xs);
+      float w_nxt = k_groups > 1 ? __ldg(ws + 1) : 0.f, x_nxt = k_groups > 1 ? __ldg(xs + SR_PAGE_ROWS) : 0.f;
       for (int kg = 0; kg < k_groups; ++kg, ++gcount) {
         const uint32_t b = gcount & 1u, par = (gcount >> 1) & 1u;
-        // weight scale x activation scale for this warpgroup's 128 tokens: one product per thread
-        if (ok) ok = mbar_wait(&sx_full[b], par, abort_flag, p.s.status);
-        comb[b * BN + e] = ok ? __ldg(scale_row + kg) * sxs[b * BN + e] : 0.f;
-        asm volatile("bar.sync %0, 128;" ::"r"(2 + wg) : "memory");
-        if (ok) ok = mbar_wait(&pfull_bar[b], par, abort_flag, p.s.status);
+        float w_far = 0.f, x_far = 0.f;
+        if (kg + 2 < k_groups) {
+          w_far = __ldg(ws + kg + 2);
+          x_far = __ldg(xs + (long long)(kg + 2) * SR_PAGE_ROWS);
+        }
+        if (ok) ok = mbar_wait_spin(&pfull_bar[b], par, abort_flag, p.s.status);
         if (ok) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t col = b * (uint32_t)BN + (uint32_t)(wg * 128);
-          const float4* cb = (const float4*)(comb + b * BN + wg * 128);        // same address in every lane
+          const float comb = w_cur * x_cur;
+          const uint32_t taddr = tmem_base + lane_off + b * (uint32_t)W8_CH + (uint32_t)(wg * 128);
           float v0[32], v1[32];
-          tmem_ld32_issue(tmem_base + lane_off + col, v0);
+          tmem_ld32_issue(taddr, v0);
 #pragma unroll
           for (int c = 0; c < 4; c += 2) {
-            tmem_ld32_issue(tmem_base + lane_off + col + (uint32_t)((c + 1) * 32), v1);
+            tmem_ld32_issue(taddr + (uint32_t)((c + 1) * 32), v1);
             tmem_wait_ld();                      // waits for both; the second is consumed after the first chunk's math
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              const float4 a = cb[c * 8 + q];
-              tot[c * 32 + 4 * q] = fmaf(a.x, v0[4 * q], tot[c * 32 + 4 * q]);
-              tot[c * 32 + 4 * q + 1] = fmaf(a.y, v0[4 * q + 1], tot[c * 32 + 4 * q + 1]);
-              tot[c * 32 + 4 * q + 2] = fmaf(a.z, v0[4 * q + 2], tot[c * 32 + 4 * q + 2]);
-              tot[c * 32 + 4 * q + 3] = fmaf(a.w, v0[4 * q + 3], tot[c * 32 + 4 * q + 3]);
-            }
-            if (c + 2 < 4) tmem_ld32_issue(tmem_base + lane_off + col + (uint32_t)((c + 2) * 32), v0);
+            for (int i = 0; i < 32; ++i) tot[c * 32 + i] = fmaf(comb, v0[i], tot[c * 32 + i]);
+            if (c + 2 < 4) tmem_ld32_issue(taddr + (uint32_t)((c + 2) * 32), v0);
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              const float4 a = cb[(c + 1) * 8 + q];
-              tot[(c + 1) * 32 + 4 * q] = fmaf(a.x, v1[4 * q], tot[(c + 1) * 32 + 4 * q]);
-              tot[(c + 1) * 32 + 4 * q + 1] = fmaf(a.y, v1[4 * q + 1], tot[(c + 1) * 32 + 4 * q + 1]);
-              tot[(c + 1) * 32 + 4 * q + 2] = fmaf(a.z, v1[4 * q + 2], tot[(c + 1) * 32 + 4 * q + 2]);
-              tot[(c + 1) * 32 + 4 * q + 3] = fmaf(a.w, v1[4 * q + 3], tot[(c + 1) * 32 + 4 * q + 3]);
-            }
+            for (int i = 0; i < 32; ++i) tot[(c + 1) * 32 + i] = fmaf(comb, v1[i], tot[(c + 1) * 32 + i]);
           }
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(&pempty_bar[b]);        // also after a failed wait: nobody is left waiting on this warp
+        w_cur = w_nxt; x_cur = x_nxt;
+        w_nxt = w_far; x_nxt = x_far;
       }
       // One decision for all eight warps (none may leave a tile alone: the other warps of its warpgroup wait for it
-      // at the named barrier of the next group): a wait that gave up anywhere in the CTA has raised the flag.
+      // at the named barriers below): a wait that gave up anywhere in the CTA has raised the flag.
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (*abort_flag) break;
-      // the tile's totals are complete: conv + SiLU on this warpgroup's two page slots
-      float cw[4] = {0.f, 0.f, 0.f, 0.f};
-      if (ch < p.n_kv) {
-        const uint2 wv = *(const uint2*)(p.conv_w + (long long)(p.n_q + ch) * SR_CONV_W);
-        const __nv_bfloat16* w4 = (const __nv_bfloat16*)&wv;
+      // The tile's totals are complete.  Two rounds of 64 channels: every thread writes its token's 64 totals as a
+      // column, then reads one channel's 64 tokens of one page slot as a row and runs conv + SiLU on them.
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        if (r) asm volatile("bar.sync %0, 128;" ::"r"(2 + wg) : "memory");     // round 0 has been read
+#pragma unroll
+        for (int c = 0; c < 64; ++c) buf[c * W8_TR_LD + tid] = tot[r * 64 + c];
+        asm volatile("bar.sync %0, 128;" ::"r"(2 + wg) : "memory");
+        const int ch_local = r * 64 + (tid & 63), ch = cb * BM + ch_local;
+        float v[64];
+        const float4* row = (const float4*)(buf + (tid & 63) * W8_TR_LD + sl * SR_PAGE_ROWS);
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+          const float4 a = row[q];
+          v[4 * q] = a.x; v[4 * q + 1] = a.y; v[4 * q + 2] = a.z; v[4 * q + 3] = a.w;
+        }
+        const __nv_bfloat16* w4 = (const __nv_bfloat16*)&cwv[r];
+        float cw[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) cw[q] = __bfloat162float(w4[q]);
-      }
-#pragma unroll
-      for (int sl = 0; sl < 2; ++sl) {
-        const int slot = SLOTS * tt + 2 * wg + sl;
         float z1, z2, z3;
-        load_history(p, false, p.s.slot_first[slot], ch, z1, z2, z3);
-        emit_slot(p, false, ch, ch_local, ct, slot, true, p.s.slot_rows[slot], tot + sl * 64, cw, z1, z2, z3);
+        load_history(p, false, first, ch, z1, z2, z3);
+        emit_slot(p, false, ch, ch_local, cb, slot, true, vr, v, cw, z1, z2, z3);
       }
     }
   }
@@ -842,7 +851,7 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
     p.k_blocks = d / (2 * BK);
     p.sx = fused.sx;
   }
-  const long long max_tiles = t_tiles * (a8 ? p.n_ct : p.n_ct + 1);
+  const long long max_tiles = a8 ? (long long)(s.max_slots / W8_SLOTS) * ((p.n_ct + 1) / 2) : t_tiles * (p.n_ct + 1);
   int grid = (int)(max_tiles < sm_count ? max_tiles : sm_count);
   if (grid < 1) grid = 1;
   if (a8) sr_proj_w8a8_kernel<<<grid, W8_THREADS, W8_SMEM_BYTES, stream>>>(map_x, map_w, p);
