@@ -322,6 +322,7 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
     fused.dump_s = nullptr;
     fused.dump_u = nullptr;
     fused.qpart = (int64_t)table->n_requests * (SR_CONV_W - 1) <= 256 ? (float*)(base + lay.off_qpart) : nullptr;
+    fused.tile_sched = base + lay.off_sched;
     fused.hist = nullptr;
     fused.in_ssm_layer = nullptr;
     fused.in_ssm_slot_stride = 0;

@@ -111,11 +111,17 @@ struct SrWorkspace {
                          // W8A8: uint8 [max_slots][64][d_model] activation codes
   size_t off_sx;         // W8A8: float [max_slots][d_model / 128][64] activation scales
   size_t off_qpart;      // float [4][256][channels] partial sums of the conv-state kernel's k quarters (small batches)
+  size_t off_sched;      // tile counter and per-pair mailboxes of the projection's tile scheduler (SR_TILE_SCHED_BYTES)
   size_t lane_bytes;     // size of one lane's block of hand-over buffers (off_kv16 .. end)
   int lanes;             // lane blocks in `total`
   size_t total;
   int64_t max_slots;
 };
+
+// The two-CTA projection hands out its tiles in index order at run time: one counter and, per CTA pair, a ring of
+// sixteen 8-byte mailboxes through which the pair's leader tells every other role of the pair which tile comes next.
+constexpr int SR_SCHED_MAX_PAIRS = 128, SR_SCHED_RING = 16;
+constexpr size_t SR_TILE_SCHED_BYTES = 256 + (size_t)SR_SCHED_MAX_PAIRS * SR_SCHED_RING * 8;
 
 static inline size_t sr_align256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -153,6 +159,7 @@ static inline SrWorkspace sr_workspace_layout(const sr_ctx* ctx, int32_t n_reque
   w.off_sx = at;        at = sr_align256(at + (ctx->w8a8 ? sizeof(float) * (size_t)w.max_slots * SR_PAGE_ROWS *
                                                                (size_t)(ctx->desc.d_model / 128) : 0));
   w.off_qpart = at;     at = sr_align256(at + ((int64_t)n_requests * (SR_CONV_W - 1) <= 256 ? sr_conv_tail_part_bytes(ctx) : 0));
+  w.off_sched = at;     at = sr_align256(at + SR_TILE_SCHED_BYTES);
   at = (at + 1023) & ~size_t(1023);
   w.lane_bytes = at - lane0;
   w.lanes = lanes < 1 ? 1 : lanes;
@@ -259,6 +266,7 @@ struct SrFused {
   __half* dump_s;    // [slot][H_v][d_k][d_v] fp16: the state entering the chunk (not written for a request's first chunk)
   __half* dump_u;    // [slot][H_v][d_v][64] fp16: the chunk's pseudo-values U^T, before the row factors
   float* qpart;      // conv state of small batches: partial sums of the batched kernel's k quarters, or null
+  void* tile_sched;  // the projection's tile scheduler state (SR_TILE_SCHED_BYTES; cleared by every launch)
 };
 
 struct SrPoolView {

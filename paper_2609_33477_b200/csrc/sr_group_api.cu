@@ -13,7 +13,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) % 16) == 
 struct GroupLayout {
   SrWorkspace base;      // header and tables as for sr_replay_states (its per-layer block is not used)
   // offsets inside one group's block of scratch; block i of a call sits at tables_end + i * block_bytes
-  size_t off_qkv16, off_zraw, off_gates, off_split, off_dump_s, off_dump_u, off_x, off_r0, off_r1, off_zg, off_y, off_hid;
+  size_t off_qkv16, off_zraw, off_gates, off_split, off_dump_s, off_dump_u, off_x, off_r0, off_r1, off_zg, off_y, off_hid, off_sched;
   size_t tables_end, block_bytes;
   int ncb;
   size_t total(int blocks) const { return tables_end + block_bytes * (size_t)blocks; }
@@ -41,6 +41,7 @@ GroupLayout group_layout(const sr_ctx* ctx, const sr_page_table* t, int32_t max_
   g.off_zg = take(rows * hv * 2);
   g.off_y = take(rows * hv * 2);
   g.off_hid = take(rows * (size_t)(max_d_ff > 0 ? max_d_ff : 0) * 2);
+  g.off_sched = take(SR_TILE_SCHED_BYTES);
   g.block_bytes = at;
   return g;
 }
@@ -169,6 +170,7 @@ int run_group(const GroupCall& c, char* ws, int32_t first_layer, int32_t n_group
   fused.kv16 = (__half*)(ws + lay.off_qkv16);
   fused.zraw = (float*)(ws + lay.off_zraw);
   fused.gates = (float*)(ws + lay.off_gates);
+  fused.tile_sched = ws + lay.off_sched;
   fused.ncb = lay.ncb;
   fused.n_kv = ctx->conv_ch;
   fused.n_gate = ctx->n_gate;

@@ -61,6 +61,8 @@ struct FusedParams {
   int32_t slot_order;    // the row operand is a packed buffer in slot order (page = slot), bf16 (group replay)
   int32_t group_t;       // token tiles per rasterisation group
   int32_t group_c;       // channel tiles (pair tiles in the two-CTA form) per block inside a group
+  unsigned int* next_tile;     // two-CTA form: tiles handed out so far beyond the first one of every pair
+  unsigned long long* mail;    // two-CTA form: [pair][SR_SCHED_RING] (sequence number << 32 | tile + 1; tile + 1 = 0: no more)
 };
 
 __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
@@ -552,6 +554,40 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 // memory and L2 traffic per flop, and room for a 6-stage ring.  The leader CTA (rank 0) issues the MMAs;
 // both CTAs run their own TMA producer and their own epilogue (the 128 channels in their tensor memory).
 
+// Tile scheduler of the two-CTA form.  Tiles are handed out in index order at run time (a pair that finishes early
+// takes the next one), so the pairs that share an anchor tile -- neighbours in the tile order -- always work on it at
+// nearly the same time, however far the pairs have drifted apart; with a fixed assignment the drift decides how often
+// the shared tile is still in L2.  The leader's producer thread draws the tile and publishes it, with its sequence
+// number, in the pair's ring of mailboxes in global memory; every other role of the pair (the partner's producer, the
+// MMA issuer, the epilogue warps of both CTAs) reads it there.  Nobody runs more than six tiles ahead of the slowest
+// role (operand ring + two accumulators), so a ring of sixteen is never overrun.
+__device__ __forceinline__ void sched_publish(unsigned long long* mail, int pair, uint32_t seq, long long tile) {
+  const unsigned long long v = ((unsigned long long)seq << 32) | (unsigned long long)(uint32_t)(tile + 1);
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(mail + (size_t)pair * SR_SCHED_RING + (seq % SR_SCHED_RING)), "l"(v) : "memory");
+}
+// the tile of sequence number seq; -1: no more tiles; -2: gave up (bounded like every wait).  Without mailboxes (a
+// launch of at most one tile per pair) the assignment is fixed: tile = pair.
+__device__ __forceinline__ long long sched_get(const unsigned long long* mail, int pair, uint32_t seq, long long total_tiles,
+                                               volatile int* abort_flag, uint32_t* status) {
+  if (!mail) return seq == 1 && pair < total_tiles ? (long long)pair : -1;
+  const unsigned long long* slot = mail + (size_t)pair * SR_SCHED_RING + (seq % SR_SCHED_RING);
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  for (;;) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(slot) : "memory");
+    if ((uint32_t)(v >> 32) == seq) return (long long)(uint32_t)v - 1;
+    if ((++spins & 0xFFu) == 0u) {
+      if (*abort_flag) return -2;
+      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        *abort_flag = 1;
+        atomicOr(status, SR_DEV_WAIT_EXPIRED);
+        return -2;
+      }
+    }
+  }
+}
+
 constexpr int STAGES2 = 6;
 constexpr int A2_BYTES = BM * BK * 2;                 // 16 KB: 128 channels of weights
 constexpr int B2_BYTES = (BN / 2) * BK * 2;           // 16 KB: 128 tokens of anchors
@@ -616,7 +652,13 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
       uint32_t phase = 0;
       bool ok = true;
       const uint64_t w_policy = l2_policy_evict_last();    // the weight block is the operand the tile order holds in L2
-      for (long long tile = pair; ok && tile < total_tiles; tile += n_pairs) {
+      long long tile = pair < total_tiles ? pair : -1;      // the leader's view; the partner reads the mailbox
+      for (uint32_t seq = 1;; ++seq) {
+        if (rank == 0 && p.mail) sched_publish(p.mail, pair, seq, ok ? tile : -1);
+        if (rank != 0 || !p.mail) tile = sched_get(p.mail, pair, seq, total_tiles, abort_flag, p.s.status);
+        if (tile < 0 || !ok) break;
+        unsigned int drawn = 0;
+        if (rank == 0 && p.mail) drawn = atomicAdd(p.next_tile, 1u);     // the tile after this one; used when this one is loaded
         int pt, tt;
         tile_coords(tile, pt, tt);
         const int slot_a = SLOTS * tt + 2 * rank;
@@ -638,6 +680,10 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
           tma_load_4d_pair(b_dst + B2_BYTES / 2, &map_x, &full_bar[stage], kb * BK, 0, p.pool_layer, page1);
           if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
         }
+        if (rank == 0 && p.mail) {
+          const long long t = (long long)drawn + n_pairs;
+          tile = t < total_tiles ? t : -1;
+        }
       }
     }
   } else if (warp == 1) {
@@ -648,7 +694,8 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
       uint32_t acc_phase = 0;
       bool ok = true;
       const uint32_t idesc = umma_idesc(2 * BM, BN, p.fp16_stage != 0);
-      for (long long tile = pair; ok && tile < total_tiles; tile += n_pairs) {
+      for (uint32_t seq = 1; ok; ++seq) {
+        if (sched_get(p.mail, pair, seq, total_tiles, abort_flag, p.s.status) < 0) break;
         if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag, p.s.status)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
@@ -675,7 +722,11 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     const int ch_local = quarter * 32 + lane;
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (long long tile = pair; tile < total_tiles; tile += n_pairs) {
+    for (uint32_t seq = 1;; ++seq) {
+      int tile_lo = 0;
+      if (lane == 0) tile_lo = (int)sched_get(p.mail, pair, seq, total_tiles, abort_flag, p.s.status);
+      const long long tile = __shfl_sync(0xffffffffu, tile_lo, 0);
+      if (tile < 0) break;
       int pt, tt;
       tile_coords(tile, pt, tt);
       const bool gate = pt == n_pt;
@@ -795,6 +846,8 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   p.gates = fused.gates;
   p.group_c = 1;
   p.group_t = 1 << 30;
+  p.next_tile = nullptr;
+  p.mail = nullptr;
 
   cudaError_t once = sr_once_per_device(SR_ONCE_PROJ_FUSED, [] {
     cudaError_t e = cudaFuncSetAttribute(sr_proj_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
@@ -820,10 +873,20 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
     const long long blocks = (c_tiles * tile_bytes + WEIGHT_BLOCK_BYTES - 1) / WEIGHT_BLOCK_BYTES;
     p.group_c = (int32_t)((c_tiles + blocks - 1) / blocks);
   }
-  auto launch_pairs = [&](const FusedParams& pp, long long pair_tiles) {
+  auto launch_pairs = [&](FusedParams pp, long long pair_tiles) {
     long long pairs = sm_count / 2;
     if (pair_tiles < pairs) pairs = pair_tiles;
+    if (pairs > SR_SCHED_MAX_PAIRS) pairs = SR_SCHED_MAX_PAIRS;
     if (pairs < 1) pairs = 1;
+    pp.next_tile = nullptr;
+    pp.mail = nullptr;
+    if (pair_tiles > pairs) {       // more than one tile per pair: tiles are handed out at run time
+      if (!fused.tile_sched) return cudaErrorInvalidValue;
+      cudaError_t e = cudaMemsetAsync(fused.tile_sched, 0, SR_TILE_SCHED_BYTES, stream);     // counter and mailboxes
+      if (e != cudaSuccess) return e;
+      pp.next_tile = (unsigned int*)fused.tile_sched;
+      pp.mail = (unsigned long long*)((char*)fused.tile_sched + 256);
+    }
     sr_proj_fused2_kernel<<<(unsigned)(2 * pairs), NUM_THREADS, SMEM2_BYTES, stream>>>(map_x, map_w, map_g, pp);
     return cudaGetLastError();
   };
