@@ -78,8 +78,8 @@ enum { SR_CONV_SILU = 0, SR_CONV_IDENTITY = 1 };  /* sr_model_desc.conv_activati
  * code = e4m3(x / s) (fp32, IEEE division, round to nearest even, saturating), and the products run on the 8-bit
  * tensor-core path; a 128-deep partial sum enters the result as weight scale x activation scale x partial sum in
  * fp32, outside the tensor core -- which is what bounds this mode: with these plain fp32 scales it runs at under
- * half of the 8-bit tensor rate, a few per cent faster than NONE on the benchmark configuration.  The gate
- * projection (bf16 weights) keeps the bf16 rows.
+ * half of the 8-bit tensor rate, as fast as NONE on the benchmark configuration.  The gate projection (bf16
+ * weights) keeps the bf16 rows.
  * W8A8 changes the VALUE computed (e4m3 keeps 4 significant bits of each activation): it is its own variant with
  * its own reference result, not an approximation of NONE held to the same tolerance. */
 enum { SR_AQ_NONE = 0, SR_AQ_E4M3_1X128 = 1 };
