@@ -118,9 +118,10 @@ struct SrWorkspace {
   int64_t max_slots;
 };
 
-// The two-CTA projection hands out its tiles in index order at run time: one counter and, per CTA pair, a ring of
-// sixteen 8-byte mailboxes through which the pair's leader tells every other role of the pair which tile comes next.
-constexpr int SR_SCHED_MAX_PAIRS = 128, SR_SCHED_RING = 16;
+// The persistent projection kernels hand out their tiles in index order at run time: one counter and, per CTA pair
+// (per CTA in the 8-bit kernel), a ring of sixteen 8-byte mailboxes through which the producer thread that draws the
+// tile tells every other role which tile comes next.
+constexpr int SR_SCHED_MAX_PAIRS = 160, SR_SCHED_RING = 16;     // pairs, or single CTAs of the 8-bit projection
 constexpr size_t SR_TILE_SCHED_BYTES = 256 + (size_t)SR_SCHED_MAX_PAIRS * SR_SCHED_RING * 8;
 
 static inline size_t sr_align256(size_t x) { return (x + 255) & ~size_t(255); }

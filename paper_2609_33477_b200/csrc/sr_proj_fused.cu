@@ -332,6 +332,41 @@ sr_proj_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   }
 }
 
+// Tile scheduler of the persistent kernels below (the two-CTA form; the 8-bit form, where a "pair" is one CTA).
+// Tiles are handed out in index order at run time (a pair that finishes early
+// takes the next one), so the pairs that share an anchor tile -- neighbours in the tile order -- always work on it at
+// nearly the same time, however far the pairs have drifted apart; with a fixed assignment the drift decides how often
+// the shared tile is still in L2.  The leader's producer thread draws the tile and publishes it, with its sequence
+// number, in the pair's ring of mailboxes in global memory; every other role of the pair (the partner's producer, the
+// MMA issuer, the epilogue warps of both CTAs) reads it there.  Nobody runs more than six tiles ahead of the slowest
+// role (operand ring + two accumulators), so a ring of sixteen is never overrun.
+__device__ __forceinline__ void sched_publish(unsigned long long* mail, int pair, uint32_t seq, long long tile) {
+  const unsigned long long v = ((unsigned long long)seq << 32) | (unsigned long long)(uint32_t)(tile + 1);
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(mail + (size_t)pair * SR_SCHED_RING + (seq % SR_SCHED_RING)), "l"(v) : "memory");
+}
+// the tile of sequence number seq; -1: no more tiles; -2: gave up (bounded like every wait).  Without mailboxes (a
+// launch of at most one tile per pair) the assignment is fixed: tile = pair.
+__device__ __forceinline__ long long sched_get(const unsigned long long* mail, int pair, uint32_t seq, long long total_tiles,
+                                               volatile int* abort_flag, uint32_t* status) {
+  if (!mail) return seq == 1 && pair < total_tiles ? (long long)pair : -1;
+  const unsigned long long* slot = mail + (size_t)pair * SR_SCHED_RING + (seq % SR_SCHED_RING);
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  for (;;) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(slot) : "memory");
+    if ((uint32_t)(v >> 32) == seq) return (long long)(uint32_t)v - 1;
+    if ((++spins & 0xFFu) == 0u) {
+      if (*abort_flag) return -2;
+      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        *abort_flag = 1;
+        atomicOr(status, SR_DEV_WAIT_EXPIRED);
+        return -2;
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------------------------
 // W8A8: e4m3 weight codes (as the caller stores them) x e4m3 activation codes (written by the quantiser, page-slot
 // order), tcgen05 kind::f8f6f4, one 128-byte row of K per stage.  Both operands carry block scales that are plain
@@ -407,7 +442,13 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      long long tile = (long long)blockIdx.x < total_tiles ? (long long)blockIdx.x : -1;
+      for (uint32_t seq = 1;; ++seq) {
+        if (p.mail) sched_publish(p.mail, blockIdx.x, seq, ok ? tile : -1);
+        else tile = sched_get(p.mail, blockIdx.x, seq, total_tiles, abort_flag, p.s.status);
+        if (tile < 0 || !ok) break;
+        unsigned int drawn = 0;
+        if (p.mail) drawn = atomicAdd(p.next_tile, 1u);            // the tile after this one
         const int tt = (int)(tile / c_tiles), ct = (int)(tile % c_tiles);
         for (int kb = 0; kb < k_groups; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, p.s.status)) { ok = false; break; }
@@ -422,13 +463,18 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
             tma_load_2d(w_dst + h * (W8_W_BYTES / 2), &map_w, &full_bar[stage], kb * W8_BK, p.w_row0 + ct * W8_CH + h * BM);
           if (++stage == W8_STAGES) { stage = 0; phase ^= 1u; }
         }
+        if (p.mail) {
+          const long long t = (long long)drawn + gridDim.x;
+          tile = t < total_tiles ? t : -1;
+        }
       }
     } else if (warp == 1 && lane == 0) {         // MMA issue
       int stage = 0;
       uint32_t phase = 0, gcount = 0;
       bool ok = true;
       const uint32_t idesc = umma_idesc_e4m3(W8_TOK, W8_CH);
-      for (long long tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      for (uint32_t seq = 1; ok; ++seq) {
+        if (sched_get(p.mail, blockIdx.x, seq, total_tiles, abort_flag, p.s.status) < 0) break;
         for (int kg = 0; kg < k_groups; ++kg, ++gcount) {
           const uint32_t b = gcount & 1u;
           // buffer b was folded two groups ago
@@ -456,7 +502,12 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     const int last_block = (p.n_q + p.n_kv - 1) / 128;     // last row of the weight-scale matrix
     uint32_t gcount = 0;
     bool ok = true;
-    for (long long tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    for (uint32_t seq = 1;; ++seq) {
+      int tile_lo = 0;
+      if (lane == 0) tile_lo = (int)sched_get(p.mail, blockIdx.x, seq, total_tiles, abort_flag, p.s.status);
+      const long long tile = __shfl_sync(0xffffffffu, tile_lo, 0);
+      // one decision for all eight warps (they meet at named barriers below, so none may leave alone)
+      if (named_bar_or(1, 256, tile == -2 || *abort_flag != 0) || tile < 0) break;
       const int tt = (int)(tile / c_tiles), ct = (int)(tile % c_tiles);
       const int cb = 2 * ct + wg;                          // this warpgroup's 128-channel block of k | v
       const float* ws = p.w_scale + (long long)min((p.n_q + cb * BM) / 128, last_block) * p.scale_ld;
@@ -509,8 +560,7 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
       }
       // One decision for all eight warps (none may leave a tile alone: the other warps of its warpgroup wait for it
       // at the named barriers below): a wait that gave up anywhere in the CTA has raised the flag.
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (*abort_flag) break;
+      if (named_bar_or(1, 256, *abort_flag != 0)) break;
       // The tile's totals are complete.  Two rounds of 64 channels: every thread writes its token's 64 totals as a
       // column, then reads one channel's 64 tokens of one page slot as a row and runs conv + SiLU on them.
 #pragma unroll
@@ -553,40 +603,6 @@ sr_proj_w8a8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 // the token operand from both shared memories, so every byte staged feeds twice the work: less shared
 // memory and L2 traffic per flop, and room for a 6-stage ring.  The leader CTA (rank 0) issues the MMAs;
 // both CTAs run their own TMA producer and their own epilogue (the 128 channels in their tensor memory).
-
-// Tile scheduler of the two-CTA form.  Tiles are handed out in index order at run time (a pair that finishes early
-// takes the next one), so the pairs that share an anchor tile -- neighbours in the tile order -- always work on it at
-// nearly the same time, however far the pairs have drifted apart; with a fixed assignment the drift decides how often
-// the shared tile is still in L2.  The leader's producer thread draws the tile and publishes it, with its sequence
-// number, in the pair's ring of mailboxes in global memory; every other role of the pair (the partner's producer, the
-// MMA issuer, the epilogue warps of both CTAs) reads it there.  Nobody runs more than six tiles ahead of the slowest
-// role (operand ring + two accumulators), so a ring of sixteen is never overrun.
-__device__ __forceinline__ void sched_publish(unsigned long long* mail, int pair, uint32_t seq, long long tile) {
-  const unsigned long long v = ((unsigned long long)seq << 32) | (unsigned long long)(uint32_t)(tile + 1);
-  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(mail + (size_t)pair * SR_SCHED_RING + (seq % SR_SCHED_RING)), "l"(v) : "memory");
-}
-// the tile of sequence number seq; -1: no more tiles; -2: gave up (bounded like every wait).  Without mailboxes (a
-// launch of at most one tile per pair) the assignment is fixed: tile = pair.
-__device__ __forceinline__ long long sched_get(const unsigned long long* mail, int pair, uint32_t seq, long long total_tiles,
-                                               volatile int* abort_flag, uint32_t* status) {
-  if (!mail) return seq == 1 && pair < total_tiles ? (long long)pair : -1;
-  const unsigned long long* slot = mail + (size_t)pair * SR_SCHED_RING + (seq % SR_SCHED_RING);
-  const long long t0 = clock64();
-  uint32_t spins = 0;
-  for (;;) {
-    unsigned long long v;
-    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(slot) : "memory");
-    if ((uint32_t)(v >> 32) == seq) return (long long)(uint32_t)v - 1;
-    if ((++spins & 0xFFu) == 0u) {
-      if (*abort_flag) return -2;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-        *abort_flag = 1;
-        atomicOr(status, SR_DEV_WAIT_EXPIRED);
-        return -2;
-      }
-    }
-  }
-}
 
 constexpr int STAGES2 = 6;
 constexpr int A2_BYTES = BM * BK * 2;                 // 16 KB: 128 channels of weights
@@ -917,7 +933,17 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   const long long max_tiles = a8 ? (long long)(s.max_slots / W8_SLOTS) * ((p.n_ct + 1) / 2) : t_tiles * (p.n_ct + 1);
   int grid = (int)(max_tiles < sm_count ? max_tiles : sm_count);
   if (grid < 1) grid = 1;
-  if (a8) sr_proj_w8a8_kernel<<<grid, W8_THREADS, W8_SMEM_BYTES, stream>>>(map_x, map_w, p);
+  if (a8) {
+    if (grid > SR_SCHED_MAX_PAIRS) grid = SR_SCHED_MAX_PAIRS;
+    if (max_tiles > grid) {         // more than one tile per CTA: tiles are handed out at run time
+      if (!fused.tile_sched) return cudaErrorInvalidValue;
+      cudaError_t e = cudaMemsetAsync(fused.tile_sched, 0, SR_TILE_SCHED_BYTES, stream);
+      if (e != cudaSuccess) return e;
+      p.next_tile = (unsigned int*)fused.tile_sched;
+      p.mail = (unsigned long long*)((char*)fused.tile_sched + 256);
+    }
+    sr_proj_w8a8_kernel<<<grid, W8_THREADS, W8_SMEM_BYTES, stream>>>(map_x, map_w, p);
+  }
   else if (scaled) sr_proj_fused_kernel<true><<<grid, NUM_THREADS_SCALED, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
   else sr_proj_fused_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
   return cudaGetLastError();
