@@ -278,6 +278,8 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
                        sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, lanes).total > workspace_bytes))
     lanes >>= 1;
   const SrWorkspace lay = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, lanes);
+  const int blocks = lanes;                                  // hand-over blocks; the streams that work on them:
+  if (lanes > SR_MAX_LANES) lanes = SR_MAX_LANES;            // (both powers of two: a block always meets the same stream)
   if (lanes > 1 && !sr_ensure_lanes(ctx)) return SR_ERR_CUDA;
 
   SrSched sched = sr_sched_view(workspace, lay, table->n_requests);
@@ -295,17 +297,76 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
                            stream) != cudaSuccess)
       return SR_ERR_CUDA;
   }
-  if (lanes > 1) {
-    if (cudaEventRecord(ctx->lane_fork, stream) != cudaSuccess) return SR_ERR_CUDA;
+  // Small batches with plain bf16 weights: the projections of up to `blocks` layers go through ONE launch on the
+  // caller's stream (a single hit would otherwise run its layers' one-wave projection launches one after the other);
+  // the rest of each layer then runs on the lanes as before.
+  const bool batched = blocks > 1 && !hooks && sr_proj_fused_batchable(ctx, lay.max_slots, sm_count);
+  const int batch_max = blocks < sr_proj_fused_batch_max() ? blocks : sr_proj_fused_batch_max();
+  auto fork = [&]() -> bool {
+    if (lanes <= 1) return true;
+    if (cudaEventRecord(ctx->lane_fork, stream) != cudaSuccess) return false;
     for (int i = 0; i < lanes - 1; ++i)
-      if (cudaStreamWaitEvent(ctx->lane_stream[i], ctx->lane_fork, 0) != cudaSuccess) return SR_ERR_CUDA;
-  }
+      if (cudaStreamWaitEvent(ctx->lane_stream[i], ctx->lane_fork, 0) != cudaSuccess) return false;
+    return true;
+  };
+  auto join = [&]() -> bool {
+    bool ok = true;
+    for (int i = 0; i < lanes - 1; ++i)
+      if (cudaEventRecord(ctx->lane_join[i], ctx->lane_stream[i]) != cudaSuccess ||
+          cudaStreamWaitEvent(stream, ctx->lane_join[i], 0) != cudaSuccess)
+        ok = false;
+    return ok;
+  };
+  if (!batched && !fork()) return SR_ERR_CUDA;
   int status = SR_OK, j = 0;
+  int projected_until = 0;            // batched: layers (by count j) whose projection has been launched
   for (int l = 0; l < d.n_layers && status == SR_OK; ++l) {
     if (!layer_mask[l]) continue;
-    const int lane = j++ % lanes;
+    if (batched && j == projected_until) {
+      // the next batch of projections: layers j .. j + n - 1 of the call, into blocks (j + i) % blocks
+      if (j > 0 && !join()) { status = SR_ERR_CUDA; break; }        // their blocks are in use until the lanes are done
+      const sr_layer_weights* bw[SR_MAX_BLOCKS];
+      int32_t bpl[SR_MAX_BLOCKS];
+      SrFused bf[SR_MAX_BLOCKS];
+      int n = 0;
+      status = SR_ERR_CUDA;
+      bool ok = true;
+      for (int l2 = l; l2 < d.n_layers && n < batch_max && ok; ++l2) {
+        if (!layer_mask[l2]) continue;
+        char* b2 = (char*)workspace + (size_t)((j + n) % blocks) * lay.lane_bytes;
+        SrFused& f = bf[n];
+        f = SrFused();
+        f.kv16 = (__half*)(b2 + lay.off_kv16);
+        f.zraw = (float*)(b2 + lay.off_zraw);
+        f.gates = (float*)(b2 + lay.off_z);
+        f.ncb = (ctx->n_k + ctx->n_v + 127) / 128;
+        f.tile_sched = b2 + lay.off_sched;
+        f.hist = nullptr;
+        if (in_conv) {
+          __nv_bfloat16* hist = (__nv_bfloat16*)(b2 + lay.off_hist);
+          SrLaunchScope scope(ctx, stream, SR_KERNEL_CONV_TAIL);
+          if (sr_launch_hist_gather(ctx, sched, (const char*)in_conv->base + (int64_t)l2 * in_conv->layer_stride_bytes,
+                                    in_conv->slot_stride_bytes, hist, stream) != cudaSuccess)
+            ok = false;
+          f.hist = hist;
+        }
+        bw[n] = &weights[l2];
+        bpl[n] = pool->layer_to_pool[l2];
+        ++n;
+      }
+      if (!ok) break;
+      {
+        SrLaunchScope scope(ctx, stream, SR_KERNEL_PROJECTION);
+        if (sr_launch_proj_fused_batch(ctx, sched, *pool, n, bpl, bw, bf, sm_count, stream) != cudaSuccess) break;
+      }
+      if (!fork()) break;
+      projected_until = j + n;
+      status = SR_OK;
+    }
+    const int lane = j % lanes;
     cudaStream_t ls = lane == 0 ? stream : ctx->lane_stream[lane - 1];
-    char* base = (char*)workspace + (size_t)lane * lay.lane_bytes;       // this lane's hand-over block
+    char* base = (char*)workspace + (size_t)(j % blocks) * lay.lane_bytes;       // this layer's hand-over block
+    ++j;
     SrFused fused;
     fused.kv16 = (__half*)(base + lay.off_kv16);
     fused.zraw = (float*)(base + lay.off_zraw);
@@ -338,7 +399,8 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
     status = SR_ERR_CUDA;       // any early exit below is a failed CUDA call; the lanes are still joined
     do {
       if (hooks && !hooks->before(hooks->user, l, pl, ls)) break;
-      if (in_conv) {
+      if (in_conv && batched) fused.hist = (__nv_bfloat16*)(base + lay.off_hist);     // gathered before the batch
+      if (in_conv && !batched) {
         __nv_bfloat16* hist = (__nv_bfloat16*)(base + lay.off_hist);
         SrLaunchScope scope(ctx, ls, SR_KERNEL_CONV_TAIL);
         if (sr_launch_hist_gather(ctx, sched, (const char*)in_conv->base + (int64_t)l * in_conv->layer_stride_bytes,
@@ -366,7 +428,7 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
         SrLaunchScope scope(ctx, ls, SR_KERNEL_WEIGHT_DECODE);
         if (sr_launch_weight_decode(ctx, weights[l], wdec, ls) != cudaSuccess) break;
       }
-      {
+      if (!batched) {
         SrLaunchScope scope(ctx, ls, SR_KERNEL_PROJECTION, ctx->w8a8 ? 2 : 1);
         if (sr_launch_proj_fused(ctx, sched, *pool, pl, weights[l], ctx->wdec_bytes ? wdec : nullptr, fused, sm_count,
                                  ls) != cudaSuccess)
@@ -392,10 +454,7 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
     } while (false);
   }
   // join: whatever happened above, `stream` resumes only after every lane's work
-  for (int i = 0; i < lanes - 1; ++i)
-    if (cudaEventRecord(ctx->lane_join[i], ctx->lane_stream[i]) != cudaSuccess ||
-        cudaStreamWaitEvent(stream, ctx->lane_join[i], 0) != cudaSuccess)
-      status = SR_ERR_CUDA;
+  if (!join()) status = SR_ERR_CUDA;
   return status;
 }
 }  // namespace

@@ -15,7 +15,8 @@
 
 #define SR_PAGE_ROWS 64
 #define SR_CONV_W 4
-#define SR_MAX_LANES 8                       // layers in flight at once on small batches
+#define SR_MAX_LANES 8                       // streams a call spreads its layers over on small batches
+#define SR_MAX_BLOCKS 32                     // blocks of per-layer hand-over buffers (layers whose buffers are alive at once)
 #define SR_LANES_BUDGET_BYTES (1024ull << 20) // ... as long as their hand-over buffers together stay below this
 
 struct sr_ctx {
@@ -168,15 +169,16 @@ static inline SrWorkspace sr_workspace_layout(const sr_ctx* ctx, int32_t n_reque
   return w;
 }
 
-// Layers in flight at once for a batch of these bounds: as many (up to SR_MAX_LANES, and no more than the model has
-// layers) as keep the hand-over buffers together within SR_LANES_BUDGET_BYTES; large batches fill the device with
+// Blocks of hand-over buffers for a batch of these bounds (layers in flight at once): as many (up to SR_MAX_BLOCKS, and
+// no more than the model has layers) as keep the blocks together within SR_LANES_BUDGET_BYTES; up to SR_MAX_LANES
+// streams work on them; large batches fill the device with
 // one layer and get one lane.  (Measured with a 24 GiB budget, i.e. two to four lanes on the 250 000-row
 // configurations, in the same run as one lane: the chunk-local kernel does run in the shared memory the next
 // layer's persistent projection leaves free, but the projection slows by as much -- steps 1.8 % and 1.0 % shorter
 // on two configurations, 1.1 % longer on the third.)
 static inline int sr_policy_lanes(const sr_ctx* ctx, int32_t n_requests, int32_t max_pages, int64_t max_total_rows) {
   const size_t per_lane = sr_workspace_layout(ctx, n_requests, max_pages, max_total_rows, 1).lane_bytes;
-  int lanes = SR_MAX_LANES;
+  int lanes = SR_MAX_BLOCKS;
   while (lanes > 1 && ((size_t)lanes * per_lane > SR_LANES_BUDGET_BYTES || lanes > ctx->desc.n_layers)) lanes >>= 1;
   return lanes;
 }
@@ -319,6 +321,12 @@ bool sr_proj_fused_exact_fp8_supported(const sr_ctx* ctx);
 cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_anchor_pool& pool, int32_t pool_layer,
                                  const sr_layer_weights& w, const void* decoded, const SrFused& fused, int sm_count,
                                  cudaStream_t stream);
+// the projections of several layers of a small batch in one launch (bf16 weights, at most one wave of tiles per layer)
+bool sr_proj_fused_batchable(const sr_ctx* ctx, int64_t max_slots, int sm_count);
+int sr_proj_fused_batch_max();
+cudaError_t sr_launch_proj_fused_batch(const sr_ctx* ctx, const SrSched& s, const sr_anchor_pool& pool, int n,
+                                       const int32_t* pool_layers, const sr_layer_weights* const* w, const SrFused* fused,
+                                       int sm_count, cudaStream_t stream);
 
 // group replay (sr_group_gemm.cu, sr_group_output.cu)
 cudaError_t sr_launch_rows_gemm(const SrSched& s, int kind, const __nv_bfloat16* a, int64_t k, const void* b, const void* b2,

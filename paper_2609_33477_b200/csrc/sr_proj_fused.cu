@@ -20,6 +20,8 @@
 // 128 x 128 block scales: 128-deep K groups are accumulated separately and added as scale x partial sum in
 // fp32 registers by eight epilogue warps (one scale per K group per tile, since a tile is one 128-channel
 // block).  sr_proj_w8a8_kernel (below) runs the 8-bit form.  All waits are bounded.
+#include <type_traits>
+
 #include "sr_umma.cuh"
 
 namespace {
@@ -610,9 +612,32 @@ constexpr int B2_BYTES = (BN / 2) * BK * 2;           // 16 KB: 128 tokens of an
 constexpr int STAGE2_BYTES = A2_BYTES + B2_BYTES;
 constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 + 256;
 
+// Several layers in ONE launch (small batches: a single hit fills the device for a fraction of one wave per layer, and
+// the launches of a call's layers would run one after the other): the tile space is (layer, channel tile, token
+// tile), layer-major, and what differs from layer to layer -- the weight and gate-weight tensor maps, the conv
+// weights, the layer's hand-over buffers, its conv history and its place in the pool -- comes from a table in the
+// kernel's parameter space.
+constexpr int PROJ_BATCH_MAX = 24;
+struct alignas(64) BatchLayer {
+  CUtensorMap map_w, map_g;
+  const __nv_bfloat16* conv_w;
+  __half* kv16;
+  float* zraw;
+  float* gates;
+  const __nv_bfloat16* hist;
+  int32_t pool_layer;
+};
+struct alignas(64) BatchTable {
+  int32_t n_layers;
+  BatchLayer layer[PROJ_BATCH_MAX];
+};
+struct NoBatch {};
+
+template <class Table>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                      const __grid_constant__ CUtensorMap map_g, const FusedParams p) {
+                      const __grid_constant__ CUtensorMap map_g, const FusedParams p, const __grid_constant__ Table bt) {
+  constexpr bool BATCHED = !std::is_same<Table, NoBatch>::value;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* full_bar = (uint64_t*)(smem + STAGES2 * STAGE2_BYTES);   // used in the leader CTA only
@@ -630,7 +655,9 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   const int n_pt = (p.n_ct + 1) / 2;              // 256-channel tiles of k | v (the last may be half empty); tile
                                                   // index n_pt is the gate tile
   const int c_tiles = p.gate_only ? 1 : n_pt + 1;
-  const long long total_tiles = (long long)t_tiles * c_tiles;
+  const long long layer_tiles = (long long)t_tiles * c_tiles;
+  long long total_tiles = layer_tiles;
+  if constexpr (BATCHED) total_tiles = layer_tiles * bt.n_layers;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES2; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
@@ -648,7 +675,12 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  auto tile_coords = [&](long long tile, int& pt, int& tt) {
+  auto tile_coords = [&](long long tile, int& layer, int& pt, int& tt) {
+    layer = 0;
+    if constexpr (BATCHED) {
+      layer = (int)(tile / layer_tiles);
+      tile -= layer * layer_tiles;
+    }
     if (p.gate_only) { pt = n_pt; tt = (int)tile; return; }
     const long long per_group = (long long)p.group_t * c_tiles;
     const int g = (int)(tile / per_group);
@@ -675,8 +707,16 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         if (tile < 0 || !ok) break;
         unsigned int drawn = 0;
         if (rank == 0 && p.mail) drawn = atomicAdd(p.next_tile, 1u);     // the tile after this one; used when this one is loaded
-        int pt, tt;
-        tile_coords(tile, pt, tt);
+        int layer, pt, tt;
+        tile_coords(tile, layer, pt, tt);
+        const CUtensorMap* mw = &map_w;
+        const CUtensorMap* mg = &map_g;
+        int pool_layer = p.pool_layer;
+        if constexpr (BATCHED) {
+          mw = &bt.layer[layer].map_w;
+          mg = &bt.layer[layer].map_g;
+          pool_layer = bt.layer[layer].pool_layer;
+        }
         const int slot_a = SLOTS * tt + 2 * rank;
         const bool by_slot = p.fp16_stage || p.slot_order;
         int page0 = by_slot ? slot_a : p.s.slot_page[slot_a], page1 = by_slot ? slot_a + 1 : p.s.slot_page[slot_a + 1];
@@ -690,10 +730,10 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
           uint8_t* a_dst = smem + stage * STAGE2_BYTES;
           uint8_t* b_dst = a_dst + A2_BYTES;
           if (rank == 0) mbar_expect_tx(&full_bar[stage], 2 * STAGE2_BYTES);     // both CTAs' loads land on this barrier
-          if (gate) tma_load_2d_pair(a_dst, &map_g, &full_bar[stage], kb * BK, rank * BM);
-          else tma_load_2d_pair_hint(a_dst, &map_w, &full_bar[stage], kb * BK, p.w_row0 + pt * 2 * BM + rank * BM, w_policy);
-          tma_load_4d_pair(b_dst, &map_x, &full_bar[stage], kb * BK, 0, p.pool_layer, page0);
-          tma_load_4d_pair(b_dst + B2_BYTES / 2, &map_x, &full_bar[stage], kb * BK, 0, p.pool_layer, page1);
+          if (gate) tma_load_2d_pair(a_dst, mg, &full_bar[stage], kb * BK, rank * BM);
+          else tma_load_2d_pair_hint(a_dst, mw, &full_bar[stage], kb * BK, p.w_row0 + pt * 2 * BM + rank * BM, w_policy);
+          tma_load_4d_pair(b_dst, &map_x, &full_bar[stage], kb * BK, 0, pool_layer, page0);
+          tma_load_4d_pair(b_dst + B2_BYTES / 2, &map_x, &full_bar[stage], kb * BK, 0, pool_layer, page1);
           if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
         }
         if (rank == 0 && p.mail) {
@@ -743,14 +783,23 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
       if (lane == 0) tile_lo = (int)sched_get(p.mail, pair, seq, total_tiles, abort_flag, p.s.status);
       const long long tile = __shfl_sync(0xffffffffu, tile_lo, 0);
       if (tile < 0) break;
-      int pt, tt;
-      tile_coords(tile, pt, tt);
+      int layer, pt, tt;
+      tile_coords(tile, layer, pt, tt);
+      FusedParams q = p;                                  // this tile's layer: its buffers, conv weights and history
+      if constexpr (BATCHED) {
+        const BatchLayer& bl = bt.layer[layer];
+        q.conv_w = bl.conv_w;
+        q.kv16 = bl.kv16;
+        q.zraw = bl.zraw;
+        q.gates = bl.gates;
+        q.hist = bl.hist;
+      }
       const bool gate = pt == n_pt;
       const int ct = 2 * pt + rank;                       // this CTA's 128-channel block
       const int ch = gate ? rank * BM + ch_local : ct * BM + ch_local;
       float cw[4] = {0.f, 0.f, 0.f, 0.f};
       if (!gate && ch < p.n_kv) {
-        const uint2 wv = *(const uint2*)(p.conv_w + (long long)(p.n_q + ch) * SR_CONV_W);
+        const uint2 wv = *(const uint2*)(q.conv_w + (long long)(p.n_q + ch) * SR_CONV_W);
         const __nv_bfloat16* e = (const __nv_bfloat16*)&wv;
 #pragma unroll
         for (int q = 0; q < 4; ++q) cw[q] = __bfloat162float(e[q]);
@@ -765,8 +814,8 @@ sr_proj_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         float v[64];
         tmem_ld32(taddr + (uint32_t)(sl * 64), v);
         tmem_ld32(taddr + (uint32_t)(sl * 64 + 32), v + 32);
-        if (sl == 0 || p.s.slot_first[slot]) load_history(p, gate, p.s.slot_first[slot], ch, z1, z2, z3);
-        emit_slot(p, gate, ch, ch_local, ct, slot, sl == 0, p.s.slot_rows[slot], v, cw, z1, z2, z3);
+        if (sl == 0 || p.s.slot_first[slot]) load_history(q, gate, p.s.slot_first[slot], ch, z1, z2, z3);
+        emit_slot(q, gate, ch, ch_local, ct, slot, sl == 0, p.s.slot_rows[slot], v, cw, z1, z2, z3);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -872,7 +921,7 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(sr_proj_w8a8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, W8_SMEM_BYTES);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(sr_proj_fused2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
+      e = cudaFuncSetAttribute(sr_proj_fused2_kernel<NoBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
     return e;
   });
   if (once != cudaSuccess) return once;
@@ -903,7 +952,7 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
       pp.next_tile = (unsigned int*)fused.tile_sched;
       pp.mail = (unsigned long long*)((char*)fused.tile_sched + 256);
     }
-    sr_proj_fused2_kernel<<<(unsigned)(2 * pairs), NUM_THREADS, SMEM2_BYTES, stream>>>(map_x, map_w, map_g, pp);
+    sr_proj_fused2_kernel<NoBatch><<<(unsigned)(2 * pairs), NUM_THREADS, SMEM2_BYTES, stream>>>(map_x, map_w, map_g, pp, NoBatch{});
     return cudaGetLastError();
   };
   if (pair_form) return launch_pairs(p, t_tiles * ((p.n_ct + 1) / 2 + 1));
@@ -946,5 +995,85 @@ cudaError_t sr_launch_proj_fused(const sr_ctx* ctx, const SrSched& s, const sr_a
   }
   else if (scaled) sr_proj_fused_kernel<true><<<grid, NUM_THREADS_SCALED, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
   else sr_proj_fused_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_x, map_w, map_g, p);
+  return cudaGetLastError();
+}
+
+// Plain bf16 weights, state-only replay, and at most one wave of pair tiles per layer: the layers of such a call go
+// through ONE launch (see BatchTable), up to sr_proj_fused_batch_max() of them at a time.
+bool sr_proj_fused_batchable(const sr_ctx* ctx, int64_t max_slots, int sm_count) {
+  if (ctx->desc.weight_format != SR_W_BF16 || ctx->fp16_stage || ctx->w8a8 || ctx->wdec_bytes) return false;
+  if (ctx->debug_flags & SR_DEBUG_SINGLE_CTA_MMA) return false;
+  const long long n_ct = (ctx->n_k + ctx->n_v + BM - 1) / BM;
+  return sm_count >= 2 && (max_slots / SLOTS) * ((n_ct + 1) / 2 + 1) <= sm_count / 2;
+}
+int sr_proj_fused_batch_max() { return PROJ_BATCH_MAX; }
+
+cudaError_t sr_launch_proj_fused_batch(const sr_ctx* ctx, const SrSched& s, const sr_anchor_pool& pool, int n,
+                                       const int32_t* pool_layers, const sr_layer_weights* const* w, const SrFused* fused,
+                                       int sm_count, cudaStream_t stream) {
+  if (n < 1 || n > PROJ_BATCH_MAX || !sr_proj_fused_batchable(ctx, s.max_slots, sm_count)) return cudaErrorInvalidValue;
+  const int d = ctx->desc.d_model;
+  const int n_kv = ctx->n_k + ctx->n_v;
+  CUtensorMap map_x;
+  if (!encode_pool_map(&map_x, pool, d, BK)) return cudaErrorInvalidValue;
+  BatchTable bt;
+  bt.n_layers = n;
+  for (int i = 0; i < n; ++i) {
+    BatchLayer& bl = bt.layer[i];
+    if (fused[i].with_q || fused[i].x_slot_order) return cudaErrorInvalidValue;
+    if (!encode_2d(&bl.map_w, w[i]->w_qkv, (uint64_t)d, (uint64_t)ctx->conv_ch, (uint64_t)d * 2, BK, BM)) return cudaErrorInvalidValue;
+    if (!encode_2d(&bl.map_g, w[i]->w_ab, (uint64_t)d, (uint64_t)ctx->n_gate, (uint64_t)d * 2, BK, BM)) return cudaErrorInvalidValue;
+    bl.conv_w = (const __nv_bfloat16*)w[i]->conv_w;
+    bl.kv16 = fused[i].kv16;
+    bl.zraw = fused[i].zraw;
+    bl.gates = fused[i].gates;
+    bl.hist = fused[i].hist;
+    bl.pool_layer = pool_layers[i];
+  }
+  FusedParams p;
+  p.s = s;
+  p.pool_layer = 0;
+  p.fp16_stage = 0;
+  p.slot_order = 0;
+  p.hist = nullptr;
+  p.conv_ch = ctx->conv_ch;
+  p.k_blocks = d / BK;
+  p.n_q = ctx->n_k;
+  p.w_row0 = ctx->n_k;
+  p.n_ct = (n_kv + BM - 1) / BM;
+  p.n_gate = ctx->n_gate;
+  p.ncb = fused[0].ncb;
+  p.n_kv = n_kv;
+  p.act_identity = ctx->desc.conv_activation == SR_CONV_IDENTITY;
+  p.w_scale = nullptr;
+  p.scale_ld = d / 128;
+  p.sx = nullptr;
+  p.gate_only = 0;
+  p.conv_w = nullptr;
+  p.kv16 = nullptr;
+  p.zraw = nullptr;
+  p.gates = nullptr;
+  p.group_c = (p.n_ct + 1) / 2 + 1;      // one block: a layer's weights are its own L2 working set
+  p.group_t = 1 << 30;
+  p.next_tile = nullptr;
+  p.mail = nullptr;
+  cudaError_t e = sr_once_per_device(SR_ONCE_PROJ_FUSED2, [] {
+    return cudaFuncSetAttribute(sr_proj_fused2_kernel<BatchTable>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES);
+  });
+  if (e != cudaSuccess) return e;
+  const long long pair_tiles = (long long)n * (s.max_slots / SLOTS) * ((p.n_ct + 1) / 2 + 1);
+  long long pairs = sm_count / 2;
+  if (pair_tiles < pairs) pairs = pair_tiles;
+  if (pairs > SR_SCHED_MAX_PAIRS) pairs = SR_SCHED_MAX_PAIRS;
+  if (pairs < 1) pairs = 1;
+  if (pair_tiles > pairs) {
+    if (!fused[0].tile_sched) return cudaErrorInvalidValue;
+    e = cudaMemsetAsync(fused[0].tile_sched, 0, SR_TILE_SCHED_BYTES, stream);
+    if (e != cudaSuccess) return e;
+    p.next_tile = (unsigned int*)fused[0].tile_sched;
+    p.mail = (unsigned long long*)((char*)fused[0].tile_sched + 256);
+  }
+  CUtensorMap unused = map_x;              // the per-layer maps come from the table
+  sr_proj_fused2_kernel<BatchTable><<<(unsigned)(2 * pairs), NUM_THREADS, SMEM2_BYTES, stream>>>(map_x, unused, unused, p, bt);
   return cudaGetLastError();
 }
