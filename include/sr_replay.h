@@ -199,9 +199,11 @@ int sr_conv_bytes_per_layer(const sr_ctx* ctx, size_t* out_bytes);
 /* Scratch bytes sr_replay_states should be given for any batch within the bounds in `table`
  * (n_requests, max_pages, max_total_rows; the pointers in `table` are not read).  The layers of one call are
  * independent of one another (every layer has its own anchors, Eq. 2), so for a batch too small to fill the GPU
- * with one layer the call runs up to eight layers side by side, each with its own block of scratch: this size
- * includes those blocks (as many as stay within 1 GiB together; one block for large batches, where keeping a
- * second layer in flight under the first one's projection measured within +-2 % of running them in turn). */
+ * with one layer the call keeps up to 32 layers in flight (on up to eight streams of the context), each with its own
+ * block of scratch: this size includes those blocks (as many of 32, 24, 16, 8, 4, 2, 1 as stay within 1 GiB together
+ * and the model has layers; one block for large batches, where keeping a second layer in flight under the first
+ * one's projection measured within +-2 % of running them in turn).  With bf16 weights such a call also runs the
+ * projections of all those layers as one launch. */
 int sr_workspace_bytes(const sr_ctx* ctx, const sr_page_table* table, size_t* out_bytes);
 
 /* The least scratch a call accepts for the same bounds: one block, layers one after the other.  A workspace

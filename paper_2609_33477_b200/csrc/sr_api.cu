@@ -276,10 +276,10 @@ int replay_impl(sr_ctx* ctx, const sr_anchor_pool* pool, const sr_page_table* ta
   int lanes = sr_policy_lanes(ctx, table->n_requests, table->max_pages, table->max_total_rows);
   while (lanes > 1 && (lanes > n_active ||
                        sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, lanes).total > workspace_bytes))
-    lanes >>= 1;
+    lanes = sr_fewer_blocks(lanes);
   const SrWorkspace lay = sr_workspace_layout(ctx, table->n_requests, table->max_pages, table->max_total_rows, lanes);
   const int blocks = lanes;                                  // hand-over blocks; the streams that work on them:
-  if (lanes > SR_MAX_LANES) lanes = SR_MAX_LANES;            // (both powers of two: a block always meets the same stream)
+  if (lanes > SR_MAX_LANES) lanes = SR_MAX_LANES;            // (the block count is a multiple: a block always meets the same stream)
   if (lanes > 1 && !sr_ensure_lanes(ctx)) return SR_ERR_CUDA;
 
   SrSched sched = sr_sched_view(workspace, lay, table->n_requests);

@@ -176,10 +176,13 @@ static inline SrWorkspace sr_workspace_layout(const sr_ctx* ctx, int32_t n_reque
 // configurations, in the same run as one lane: the chunk-local kernel does run in the shared memory the next
 // layer's persistent projection leaves free, but the projection slows by as much -- steps 1.8 % and 1.0 % shorter
 // on two configurations, 1.1 % longer on the third.)
+// the block counts a call may use: 32, 24, 16, 8, 4, 2, 1 (all multiples of the stream count they are served by, so a
+// block always meets the same stream)
+static inline int sr_fewer_blocks(int blocks) { return blocks == 32 ? 24 : (blocks == 24 ? 16 : blocks >> 1); }
 static inline int sr_policy_lanes(const sr_ctx* ctx, int32_t n_requests, int32_t max_pages, int64_t max_total_rows) {
   const size_t per_lane = sr_workspace_layout(ctx, n_requests, max_pages, max_total_rows, 1).lane_bytes;
   int lanes = SR_MAX_BLOCKS;
-  while (lanes > 1 && ((size_t)lanes * per_lane > SR_LANES_BUDGET_BYTES || lanes > ctx->desc.n_layers)) lanes >>= 1;
+  while (lanes > 1 && ((size_t)lanes * per_lane > SR_LANES_BUDGET_BYTES || lanes > ctx->desc.n_layers)) lanes = sr_fewer_blocks(lanes);
   return lanes;
 }
 
