@@ -514,3 +514,27 @@ def test_a_request_gets_the_same_bits_alone_and_in_a_large_batch(name):
         torch.cuda.synchronize()
         assert torch.equal(rep1.out_conv[0], rep.out_conv[i]) and torch.equal(rep1.out_ssm[0], rep.out_ssm[i])
         rep1.close()
+
+
+def test_layers_projected_in_one_launch_match_layers_projected_alone():
+    """A small batch with bf16 weights runs the projections of all its layers as one launch; a call that rebuilds a
+    single layer runs that layer's own launch.  Tile for tile the arithmetic is the same, so both states of every
+    layer are bit-identical (a comparison of the CUDA path with itself; `layers_small` is compared with the oracle
+    in the named-workload test)."""
+    import dataclasses
+    wl = synth.build_workload("layers_small", device="cuda")
+    rep = B.Replayer(wl)
+    rep.replay_states()
+    torch.cuda.synchronize()
+    assert rep.device_status() == 0
+    n = len(wl.layer_mask)
+    for l in (0, 4, n - 1):
+        one = dataclasses.replace(wl, layer_mask=[1 if j == l else 0 for j in range(n)])
+        rep1 = B.Replayer(one)
+        rep1.replay_states()
+        torch.cuda.synchronize()
+        assert rep1.device_status() == 0
+        assert torch.equal(rep1.out_ssm[:, l], rep.out_ssm[:, l]) and torch.equal(rep1.out_conv[:, l], rep.out_conv[:, l])
+        assert rep1.last_launch_count() < rep.last_launch_count()
+        rep1.close()
+    rep.close()
