@@ -156,3 +156,28 @@ def test_group_replay_checks_its_arguments_on_the_host(lib):
     assert lib.sr_workspace_bytes(odd, C.byref(table), C.byref(n)) == B.SR_OK
     assert lib.sr_group_workspace_bytes(odd, C.byref(table), 0, C.byref(n)) == B.SR_ERR_UNSUPPORTED_SHAPE
     B.sr_destroy(odd)
+
+
+def test_recommended_workspace_holds_a_block_per_layer_in_flight(lib):
+    """sr_workspace_bytes = the tables + N blocks of per-layer hand-over buffers, N the largest of 32, 24, 16, 8, 4, 2, 1
+    that the model has layers for and that stays within 1 GiB; sr_workspace_bytes_min = the tables + one block."""
+    table = B.sr_page_table(None, None, 1, 8, 512, 512)            # one hit of 512 anchors
+    sizes = {}
+    for n_layers in (1, 2, 3, 8, 23, 24, 31, 32, 48):
+        ctx = B.sr_create(_desc(n_layers=n_layers))
+        one, rec = B.sr_workspace_bytes_min(ctx, table), B.sr_workspace_bytes(ctx, table)
+        sizes[n_layers] = (one, rec)
+        B.sr_destroy(ctx)
+    one = sizes[1][0]
+    assert sizes[1][1] == one
+    block = sizes[2][1] - one                                      # two blocks - one block
+    assert block > 0 and all(s[0] == one for s in sizes.values())
+    expect = {1: 1, 2: 2, 3: 2, 8: 8, 23: 16, 24: 24, 31: 24, 32: 32, 48: 32}
+    for n_layers, blocks in expect.items():
+        assert sizes[n_layers][1] == one + (blocks - 1) * block, n_layers
+    # a batch whose blocks would pass 1 GiB together gets fewer of them
+    big = B.sr_page_table(None, None, 64, 128, 8192, 64 * 8192)
+    ctx = B.sr_create(_desc(n_layers=32, d_model=5120, n_k_heads=16, n_v_heads=32))
+    one_big, rec_big = B.sr_workspace_bytes_min(ctx, big), B.sr_workspace_bytes(ctx, big)
+    assert rec_big == one_big and one_big > (1 << 30)
+    B.sr_destroy(ctx)
